@@ -1,0 +1,171 @@
+"""CPU oracle for the value-driven memory — TEST INFRASTRUCTURE, not the product.
+
+A ctypes front for ``evk_oracle.c`` (plain C, fp64): exact two-phase retrieval
+(Section 3.2) and the unified value update (Eq. 4 / Eq. 8).  Only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import this package; it
+imports nothing from the CUDA package and is never given a value that came from
+it.  Inputs are numpy arrays; embeddings and queries are bfloat16 bit patterns
+held as ``uint16``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "evk_oracle.c")
+_LIB = os.path.join(_HERE, "libevk_oracle.so")
+
+_CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+           "-ffp-contract=off", "-fno-fast-math", "-fexcess-precision=standard"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc if the shared object is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    subprocess.run(["gcc", *_CFLAGS, "-o", tmp, _SRC, "-lm"], check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    c_i32, c_i64, c_f32, c_f64 = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_double
+    p = ctypes.c_void_p
+    lib.evk_oracle_bf16_round.argtypes = [p, p, c_i64]
+    lib.evk_oracle_bf16_round.restype = None
+    lib.evk_oracle_bf16_decode.argtypes = [p, p, c_i64]
+    lib.evk_oracle_bf16_decode.restype = None
+    lib.evk_oracle_threads.argtypes = []
+    lib.evk_oracle_threads.restype = ctypes.c_int
+    lib.evk_oracle_sims.argtypes = [p, c_i64, c_i32, p, p]
+    lib.evk_oracle_sims.restype = None
+    lib.evk_oracle_phase1.argtypes = [p, c_i64, c_i32, p, c_i32, p, p]
+    lib.evk_oracle_phase1.restype = c_i32
+    lib.evk_oracle_phase2.argtypes = [p, p, c_i32, p, c_f64, c_i32, p, p]
+    lib.evk_oracle_phase2.restype = c_i32
+    lib.evk_oracle_q_update_f64.argtypes = [p, p, p, c_i64, c_f64]
+    lib.evk_oracle_q_update_f64.restype = None
+    lib.evk_oracle_q_update_f32.argtypes = [p, p, p, c_i64, c_f32]
+    lib.evk_oracle_q_update_f32.restype = None
+    _lib = lib
+    return lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def threads() -> int:
+    """Host threads the similarity scan spreads bank rows over."""
+    return int(_load().evk_oracle_threads())
+
+
+def bf16_round(x) -> np.ndarray:
+    """fp32 -> bfloat16 bits, round to nearest even (the insert boundary)."""
+    x = _c(x, np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    _load().evk_oracle_bf16_round(_ptr(x), _ptr(out), x.size)
+    return out
+
+
+def bf16_decode(bits) -> np.ndarray:
+    """bfloat16 bits -> fp64, exact."""
+    bits = _c(bits, np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().evk_oracle_bf16_decode(_ptr(bits), _ptr(out), bits.size)
+    return out
+
+
+def sims(bank_bits, query_bits) -> np.ndarray:
+    """Inner products of one query with every bank row, fp64 (phase 1 scores)."""
+    bank_bits = _c(bank_bits, np.uint16)
+    query_bits = _c(query_bits, np.uint16)
+    size, d = bank_bits.shape
+    assert query_bits.shape == (d,)
+    out = np.empty(size, dtype=np.float64)
+    _load().evk_oracle_sims(_ptr(bank_bits), size, d, _ptr(query_bits), _ptr(out))
+    return out
+
+
+def phase1(bank_bits, query_bits, k1: int):
+    """Top-k1 pool per query by (similarity desc, id asc): ids int32, sims fp64."""
+    bank_bits = _c(bank_bits, np.uint16)
+    query_bits = _c(query_bits, np.uint16)
+    if query_bits.ndim == 1:
+        query_bits = query_bits[None, :]
+    size, d = bank_bits.shape
+    b = query_bits.shape[0]
+    assert query_bits.shape[1] == d
+    ids = np.empty((b, k1), dtype=np.int32)
+    sm = np.empty((b, k1), dtype=np.float64)
+    lib = _load()
+    for i in range(b):
+        lib.evk_oracle_phase1(_ptr(bank_bits), size, d, _ptr(query_bits[i]), k1,
+                              _ptr(ids[i]), _ptr(sm[i]))
+    return ids, sm
+
+
+def phase2(pool_ids, pool_sims, q_stage, w: float, k2: int):
+    """Cut each pool to k2 by (1-w)*sim + w*Q (score desc, sim desc, id asc)."""
+    pool_ids = _c(pool_ids, np.int32)
+    pool_sims = _c(pool_sims, np.float64)
+    q_stage = _c(q_stage, np.float32)
+    if pool_ids.ndim == 1:
+        pool_ids, pool_sims = pool_ids[None, :], pool_sims[None, :]
+    b, k1 = pool_ids.shape
+    ids = np.empty((b, k2), dtype=np.int32)
+    sc = np.empty((b, k2), dtype=np.float64)
+    lib = _load()
+    for i in range(b):
+        lib.evk_oracle_phase2(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage),
+                              float(w), k2, _ptr(ids[i]), _ptr(sc[i]))
+    return ids, sc
+
+
+def retrieve(bank_bits, query_bits, q_stage, k1: int, k2: int, w: float):
+    """Both phases; returns (ids, scores, pool_ids, pool_sims)."""
+    pool_ids, pool_sims = phase1(bank_bits, query_bits, k1)
+    ids, sc = phase2(pool_ids, pool_sims, q_stage, w, k2)
+    return ids, sc, pool_ids, pool_sims
+
+
+def q_update_f64(q_stage, ids, rewards, alpha: float) -> np.ndarray:
+    """Eq. 4 applied in array order, fp64; returns the new table (input untouched)."""
+    q = np.array(q_stage, dtype=np.float64, order="C", copy=True)
+    ids = _c(ids, np.int32)
+    rewards = _c(rewards, np.float32)
+    assert ids.shape == rewards.shape and ids.ndim == 1
+    if ids.size:
+        assert ids.min() >= 0 and ids.max() < q.size
+    _load().evk_oracle_q_update_f64(_ptr(q), _ptr(ids), _ptr(rewards), ids.size, float(alpha))
+    return q
+
+
+def q_update_f32(q_stage, ids, rewards, alpha) -> np.ndarray:
+    """Eq. 4 in binary32, three separately rounded operations per step, array order."""
+    q = np.array(q_stage, dtype=np.float32, order="C", copy=True)
+    ids = _c(ids, np.int32)
+    rewards = _c(rewards, np.float32)
+    assert ids.shape == rewards.shape and ids.ndim == 1
+    if ids.size:
+        assert ids.min() >= 0 and ids.max() < q.size
+    _load().evk_oracle_q_update_f32(_ptr(q), _ptr(ids), _ptr(rewards), ids.size,
+                                    float(np.float32(alpha)))
+    return q

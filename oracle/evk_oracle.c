@@ -1,0 +1,174 @@
+/*
+ * evk_oracle.c — TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, fp64 CPU statement of what the value-driven memory computes:
+ * the two-phase retrieval of Section 3.2 ("Memory Architecture and Value-Driven
+ * Retrieval") and the unified value update of Eq. 4 (restated as Eq. 8 in
+ * Appendix A).  Only the tests, the smoke check and the benchmark's CPU-baseline
+ * leg may call it.  It shares no code with the CUDA library and never sees a
+ * value the CUDA library produced.
+ *
+ * Stored embeddings and queries are bfloat16 bit patterns (uint16_t); they are
+ * widened to fp64 exactly, so every product below is exact and every sum is a
+ * plain left-to-right fp64 sum over the embedding dimension.
+ *
+ * Every function here is pinned by tests/test_oracle_*.py against closed forms,
+ * invariants, library routines and brute force; none is "parity unpinned" except
+ * the general mixing weight 0 < w < 1 of evk_oracle_phase2, whose formula is a
+ * reading (the paper's own rule is w = 1) and is pinned only through its special
+ * cases, a hand-worked exact example and monotonicity.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- bfloat16 <-> IEEE ------------------------------------------------- */
+
+/* bfloat16 is the upper half of an IEEE binary32; widening is exact. */
+static double bf16_to_f64(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Round-to-nearest-even narrowing of binary32 to bfloat16 (the storage
+ * precision of the bank; the rounding is part of the insert boundary). */
+static uint16_t f32_to_bf16(float x) {
+    uint32_t u;
+    memcpy(&u, &x, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) /* NaN: keep sign, force quiet */
+        return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+void evk_oracle_bf16_round(const float *x, uint16_t *out, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) out[i] = f32_to_bf16(x[i]);
+}
+
+void evk_oracle_bf16_decode(const uint16_t *bits, double *out, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) out[i] = bf16_to_f64(bits[i]);
+}
+
+int evk_oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---- Phase 1: dense retrieval (Section 3.2) ----------------------------- */
+
+/* sim[i] = <q, e_i> for every stored entry i < size.  Rows are independent, so
+ * they may be spread over host threads; each row's sum is sequential. */
+void evk_oracle_sims(const uint16_t *bank, int64_t size, int32_t d,
+                     const uint16_t *query, double *sims) {
+    double *q = (double *)malloc((size_t)d * sizeof(double));
+    for (int32_t j = 0; j < d; ++j) q[j] = bf16_to_f64(query[j]);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < size; ++i) {
+        const uint16_t *e = bank + i * (int64_t)d;
+        double acc = 0.0;
+        for (int32_t j = 0; j < d; ++j) acc += q[j] * bf16_to_f64(e[j]);
+        sims[i] = acc;
+    }
+    free(q);
+}
+
+typedef struct {
+    double key;  /* primary, descending   */
+    double key2; /* secondary, descending */
+    int32_t id;  /* last, ascending       */
+} ranked_t;
+
+static int ranked_cmp(const void *a, const void *b) {
+    const ranked_t *x = (const ranked_t *)a, *y = (const ranked_t *)b;
+    if (x->key > y->key) return -1;
+    if (x->key < y->key) return 1;
+    if (x->key2 > y->key2) return -1;
+    if (x->key2 < y->key2) return 1;
+    return (x->id > y->id) - (x->id < y->id);
+}
+
+/* The top-K candidate pool C(x): all `size` similarities, fully sorted by
+ * (similarity descending, id ascending); the first min(k1, size) are the pool.
+ * Unused slots get id -1 and similarity -inf.  Returns the pool length. */
+int32_t evk_oracle_phase1(const uint16_t *bank, int64_t size, int32_t d,
+                          const uint16_t *query, int32_t k1,
+                          int32_t *pool_ids, double *pool_sims) {
+    int32_t n_pool = (int32_t)((int64_t)k1 < size ? (int64_t)k1 : size);
+    for (int32_t j = 0; j < k1; ++j) { pool_ids[j] = -1; pool_sims[j] = -INFINITY; }
+    if (size <= 0) return 0;
+    double *sims = (double *)malloc((size_t)size * sizeof(double));
+    ranked_t *r = (ranked_t *)malloc((size_t)size * sizeof(ranked_t));
+    evk_oracle_sims(bank, size, d, query, sims);
+    for (int64_t i = 0; i < size; ++i) { r[i].key = sims[i]; r[i].key2 = 0.0; r[i].id = (int32_t)i; }
+    qsort(r, (size_t)size, sizeof(ranked_t), ranked_cmp);
+    for (int32_t j = 0; j < n_pool; ++j) { pool_ids[j] = r[j].id; pool_sims[j] = r[j].key; }
+    free(r);
+    free(sims);
+    return n_pool;
+}
+
+/* ---- Phase 2: value filter (Section 3.2) -------------------------------- */
+
+/* The pool is cut down to the final k2 items with the stage's value estimates.
+ * score = (1-w)*sim + w*Q_stage[id]; w = 1 is the paper's rule (rank by Q alone),
+ * w = 0 its similarity-only ablation arm.  Order: (score desc, sim desc, id asc).
+ * q_stage is the fp32 value table of ONE stage, widened exactly.  Pool slots with
+ * id < 0 are padding and are ignored.  Unused outputs get id -1, score -inf. */
+int32_t evk_oracle_phase2(const int32_t *pool_ids, const double *pool_sims, int32_t k1,
+                          const float *q_stage, double w, int32_t k2,
+                          int32_t *ids_out, double *scores_out) {
+    ranked_t *r = (ranked_t *)malloc((size_t)(k1 > 0 ? k1 : 1) * sizeof(ranked_t));
+    int32_t n = 0;
+    for (int32_t j = 0; j < k1; ++j) {
+        if (pool_ids[j] < 0) continue;
+        double qv = (double)q_stage[pool_ids[j]];
+        r[n].key = (1.0 - w) * pool_sims[j] + w * qv;
+        r[n].key2 = pool_sims[j];
+        r[n].id = pool_ids[j];
+        ++n;
+    }
+    qsort(r, (size_t)n, sizeof(ranked_t), ranked_cmp);
+    int32_t n_out = n < k2 ? n : k2;
+    for (int32_t j = 0; j < k2; ++j) { ids_out[j] = -1; scores_out[j] = -INFINITY; }
+    for (int32_t j = 0; j < n_out; ++j) { ids_out[j] = r[j].id; scores_out[j] = r[j].key; }
+    free(r);
+    return n_out;
+}
+
+/* ---- Eq. 4: unified value update ---------------------------------------- */
+
+/* Q <- Q + alpha*(r - Q) for each (id, reward) strictly in array order, on one
+ * stage's table.  fp64 truth. */
+void evk_oracle_q_update_f64(double *q_stage, const int32_t *ids, const float *rewards,
+                             int64_t m, double alpha) {
+    for (int64_t t = 0; t < m; ++t) {
+        double q = q_stage[ids[t]];
+        q_stage[ids[t]] = q + alpha * ((double)rewards[t] - q);
+    }
+}
+
+/* The same recurrence in binary32: a subtraction, a multiplication and an
+ * addition, each rounded to nearest on its own (this file is compiled with
+ * -ffp-contract=off; the volatile temporaries also keep x87-style excess
+ * precision and fusing out).  This is the bit-level definition of the stored
+ * table after a batch. */
+void evk_oracle_q_update_f32(float *q_stage, const int32_t *ids, const float *rewards,
+                             int64_t m, float alpha) {
+    for (int64_t t = 0; t < m; ++t) {
+        volatile float q = q_stage[ids[t]];
+        volatile float diff = rewards[t] - q;
+        volatile float step = alpha * diff;
+        volatile float next = q + step;
+        q_stage[ids[t]] = next;
+    }
+}
