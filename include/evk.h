@@ -1,0 +1,181 @@
+/*
+ * evk.h — C ABI of the value-driven experience memory (CUDA, sm_100a).
+ *
+ * The library keeps a bank of embeddings with one value estimate per entry and
+ * stage, and runs the two operations of the method on it:
+ *   - value-driven retrieval (Section 3.2): dense retrieval of a top-k1 candidate
+ *     pool by inner-product similarity, then a cut to k2 items using the
+ *     stage-specific value table Q_stage;
+ *   - the unified value update (Eq. 4; Eq. 8 in Appendix A):
+ *     Q <- Q + alpha * (r - Q) for every retrieved item once a reward is seen.
+ * New experiences are appended as the memory grows (Eq. 1).
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless its name ends in `_host`.
+ *     The caller owns all device memory (bank arena, workspaces, inputs,
+ *     outputs); the library allocates none and frees none.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *     return; work is ordered by the stream, so an insert or update enqueued
+ *     before a retrieve on the same stream is visible to it.  Calls on one handle
+ *     from several streams or threads at once are not synchronised.
+ *   - Every function returning int returns EVK_OK (0) or a negative evk_status.
+ *     Errors detectable on the host are returned before anything is enqueued.
+ *     Errors only the device can see (an id out of range, a non-finite reward, a
+ *     wait that ran out) are recorded in a device status word by a checking pass
+ *     that runs before any mutation; the mutating kernels of that call then do
+ *     nothing.  evk_last_status() reads the word.
+ *   - No function throws, aborts or traps.
+ */
+#ifndef EVK_H_
+#define EVK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum evk_status {
+    EVK_OK = 0,
+    EVK_ERR_INVALID = -1,        /* bad argument (null pointer, stage, k, alpha, w, dtype, alignment) */
+    EVK_ERR_CAPACITY = -2,       /* insert beyond the capacity given at create                       */
+    EVK_ERR_WORKSPACE = -3,      /* workspace or arena smaller than the *_bytes query says            */
+    EVK_ERR_RANGE = -4,          /* device check: an entry id outside [0, size)                       */
+    EVK_ERR_NONFINITE = -5,      /* device check: a reward that is NaN or infinite                    */
+    EVK_ERR_DEVICE_TIMEOUT = -6, /* device: a bounded wait inside a kernel ran out                    */
+    EVK_ERR_CUDA = -7,           /* a CUDA runtime or driver call failed                              */
+    EVK_ERR_UNSUPPORTED = -8     /* shape outside what the kernels support (see each call)            */
+} evk_status;
+
+enum { EVK_DTYPE_F32 = 0, EVK_DTYPE_BF16 = 1 };
+enum { EVK_STAGE_DRAFT = 0, EVK_STAGE_REFINE = 1, EVK_STAGE_ALL = -1 };
+/* Which phase-1 kernel evk_retrieve uses. */
+enum { EVK_SCORING_AUTO = 0, EVK_SCORING_STREAM = 1, EVK_SCORING_TENSOR = 2 };
+
+enum { EVK_MAX_K1 = 1024, EVK_MAX_D = 2048, EVK_MAX_STAGES = 8 };
+
+typedef struct evk_mem evk_mem; /* opaque; host-side state only */
+
+typedef struct evk_config {
+    int32_t d;          /* embedding width; multiple of 8, <= EVK_MAX_D                    */
+    int32_t n_stages;   /* value tables per entry; 2 = {draft, refine} (Appendix A)          */
+    int64_t capacity;   /* most entries the bank will ever hold, < 2^31                      */
+    float q_default;    /* value given to stages an insert does not name                     */
+    int32_t reserved;   /* must be 0                                                         */
+    void *arena;        /* device memory, 256-byte aligned, evk_mem_bytes_required() bytes   */
+    size_t arena_bytes;
+} evk_config;
+
+/* Bytes of device memory a bank of this shape needs (embeddings as bf16 rows
+ * [capacity][d], value tables fp32 [n_stages][capacity], a status word).  0 if the
+ * config is invalid.  `arena` and `arena_bytes` are ignored. */
+size_t evk_mem_bytes_required(const evk_config *cfg);
+
+/* Create an empty memory M_0 over the caller's arena (Eq. 1 starts from a seed
+ * bank; seed entries are inserted like any other).  The arena is not cleared
+ * except for the status word (one small async memset on the default stream,
+ * followed by a synchronise).  The handle is host memory owned by the library
+ * until evk_mem_destroy. */
+int evk_mem_create(const evk_config *cfg, evk_mem **out);
+
+/* Free the host-side handle.  Device memory stays the caller's. */
+int evk_mem_destroy(evk_mem *mem);
+
+/* Entries currently stored (host-side count, already including inserts that are
+ * enqueued but not yet executed). */
+int64_t evk_mem_size(const evk_mem *mem);
+
+/* Choose the phase-1 kernel: AUTO (default) picks by batch size and shape,
+ * STREAM forces the streaming kernel, TENSOR the tcgen05 kernel (retrieve then
+ * returns EVK_ERR_UNSUPPORTED for shapes that kernel cannot take). */
+int evk_mem_set_scoring(evk_mem *mem, int mode);
+
+/* Append n entries: M <- M ∪ {new items} (Eq. 1).  `emb` is [n][d] row-major,
+ * fp32 (rounded to bf16, nearest-even) or bf16 (copied).  Entry ids are the
+ * insertion indices size, size+1, ...; they are written to ids_out [n] if it is
+ * not NULL.  `q_init` [n] (or NULL for q_default) seeds the value table of
+ * `stage`, or of every stage with EVK_STAGE_ALL; other stages get q_default.
+ * Embeddings are stored as given: the library does not normalise them.
+ * Errors: EVK_ERR_CAPACITY (nothing is inserted), EVK_ERR_INVALID. */
+int evk_mem_insert(evk_mem *mem, const void *emb, int emb_dtype, int64_t n, int stage,
+                   const float *q_init, int32_t *ids_out, void *stream);
+
+/* Workspace bytes evk_retrieve needs for a batch of B queries and pool size k1
+ * at the bank's capacity (an upper bound for every size up to capacity). */
+size_t evk_retrieve_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1);
+
+/* Value-driven retrieval (Section 3.2) for B queries at one stage.
+ *   phase 1: sim[b][i] = <query_b, e_i> (bf16 operands, fp32 accumulation) over
+ *            all stored entries; the pool is the k1 entries of largest sim,
+ *            ordered (sim descending, id ascending);
+ *   phase 2: score = (1-w)*sim + w*Q_stage[id] over the pool; the result is the k2
+ *            entries of largest score, ordered (score desc, sim desc, id asc).
+ *            w = 1 ranks the pool by Q_stage alone, which is the rule the method
+ *            states; w = 0 is similarity-only retrieval.
+ * queries: [B][d] row-major, fp32 (rounded to bf16 first) or bf16.
+ * ids_out [B][k2] int32, scores_out [B][k2] fp32; pool_ids_out / pool_sims_out
+ * [B][k1] may be NULL.  If fewer than k1 (k2) entries exist, the pool (result) is
+ * padded with id -1 and score -inf; an empty bank is not an error.
+ * Limits: 1 <= k2 <= k1 <= EVK_MAX_K1, 0 <= w <= 1, B >= 0.
+ * The workspace must hold evk_retrieve_workspace_bytes(mem, B, k1) bytes, 256-byte
+ * aligned; its contents are scratch and calls sharing one workspace must not
+ * overlap on the device. */
+int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage,
+                 int32_t k1, int32_t k2, float w,
+                 int32_t *ids_out, float *scores_out,
+                 int32_t *pool_ids_out, float *pool_sims_out,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace bytes evk_q_update needs for a batch of M updates. */
+size_t evk_q_update_workspace_bytes(const evk_mem *mem, int64_t M);
+
+/* Unified value update (Eq. 4): for t = 0..M-1 in array order,
+ *   Q_stage[ids[t]] <- Q + alpha * (rewards[t] - Q)
+ * in binary32 as a subtraction, a multiplication and an addition, each rounded to
+ * nearest on its own (no fused multiply-add).  An id that occurs several times
+ * receives its updates one after another in array order, so the stored bits equal
+ * those of the sequential loop and do not depend on how the batch is split across
+ * calls.  0 < alpha <= 1.  Ids outside [0, size) or non-finite rewards make the
+ * whole call a no-op and set the status word (EVK_ERR_RANGE / EVK_ERR_NONFINITE).
+ * The workspace must hold evk_q_update_workspace_bytes(mem, M) bytes. */
+int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
+                 const float *rewards, float alpha,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* Copy Q_stage[first .. first+n) to / from a device array. */
+int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream);
+int evk_q_write(evk_mem *mem, int stage, int64_t first, int64_t n, const float *values, void *stream);
+
+/* Copy the stored bf16 rows [first .. first+n) to a device array [n][d] of uint16. */
+int evk_bank_read(evk_mem *mem, int64_t first, int64_t n, void *out_bf16, void *stream);
+
+/* Host-buffer forms of the two hot calls, for callers whose data lives in host
+ * memory (pinned memory makes the copies asynchronous).  They copy the inputs to
+ * the device, run the same kernels, copy the results back and synchronise the
+ * stream before returning.  `workspace` must hold the *_host_workspace_bytes
+ * amount (device memory: staging plus the kernel workspace). */
+size_t evk_retrieve_host_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1, int32_t k2);
+int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32_t B, int stage,
+                      int32_t k1, int32_t k2, float w,
+                      int32_t *ids_out_host, float *scores_out_host,
+                      void *workspace, size_t workspace_bytes, void *stream);
+size_t evk_q_update_host_workspace_bytes(const evk_mem *mem, int64_t M);
+int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stage,
+                      const float *rewards_host, float alpha,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Synchronise `stream`, return the device status word (EVK_OK or the first
+ * device-detected error since the last read) and clear it. */
+int evk_last_status(evk_mem *mem, void *stream);
+
+/* Number of kernels this handle has launched so far (host-side counter). */
+int64_t evk_launch_count(const evk_mem *mem);
+
+/* A static, human-readable name for a status code. */
+const char *evk_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EVK_H_ */

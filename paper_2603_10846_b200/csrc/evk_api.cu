@@ -1,0 +1,330 @@
+// The C ABI (include/evk.h): argument checks, memory layout, kernel dispatch.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "evk_common.cuh"
+#include "evk_kernels.cuh"
+
+using namespace evk;
+
+struct evk_mem {
+    evk_config cfg;
+    int64_t size;
+    __nv_bfloat16 *bank;  // [capacity][d]
+    float *q_tables;      // [n_stages][capacity]
+    int32_t *status;      // device status word
+    int scoring;
+    int64_t launches;
+};
+
+namespace {
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct ArenaLayout {
+    size_t bank, q_tables, status, total;
+};
+
+bool config_ok(const evk_config *c) {
+    return c && c->d > 0 && c->d % 8 == 0 && c->d <= EVK_MAX_D && c->n_stages >= 1 &&
+           c->n_stages <= EVK_MAX_STAGES && c->capacity >= 1 && c->capacity < ((int64_t)1 << 31) &&
+           c->reserved == 0 && isfinite(c->q_default);
+}
+
+ArenaLayout arena_layout(const evk_config *c) {
+    ArenaLayout l;
+    l.bank = 0;
+    l.q_tables = align256((size_t)c->capacity * c->d * sizeof(__nv_bfloat16));
+    l.status = l.q_tables + align256((size_t)c->n_stages * c->capacity * sizeof(float));
+    l.total = l.status + 256;
+    return l;
+}
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+struct RetrieveLayout {
+    size_t q_bf16, pool_ids, pool_sims, part_counts, part_keys, total;
+    int nparts_max;
+};
+
+RetrieveLayout retrieve_layout(const evk_mem *m, int32_t B, int32_t k1) {
+    RetrieveLayout l;
+    const size_t b = (size_t)(B > 0 ? B : 0);
+    const StreamPlan plan = stream_plan(m->cfg.capacity, m->cfg.d, B, k1);
+    l.nparts_max = plan.nparts;
+    l.q_bf16 = 0;
+    l.pool_ids = l.q_bf16 + align256(b * m->cfg.d * sizeof(__nv_bfloat16));
+    l.pool_sims = l.pool_ids + align256(b * k1 * sizeof(int32_t));
+    l.part_counts = l.pool_sims + align256(b * k1 * sizeof(float));
+    l.part_keys = l.part_counts + align256(b * l.nparts_max * sizeof(int));
+    l.total = l.part_keys + align256(b * l.nparts_max * (size_t)k1 * sizeof(uint64_t));
+    return l;
+}
+
+bool stage_ok(const evk_mem *m, int stage) { return stage >= 0 && stage < m->cfg.n_stages; }
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? EVK_OK : EVK_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+size_t evk_mem_bytes_required(const evk_config *cfg) {
+    if (!config_ok(cfg)) return 0;
+    return arena_layout(cfg).total;
+}
+
+int evk_mem_create(const evk_config *cfg, evk_mem **out) {
+    if (!out) return EVK_ERR_INVALID;
+    *out = nullptr;
+    if (!config_ok(cfg) || !cfg->arena || !aligned(cfg->arena, 256)) return EVK_ERR_INVALID;
+    const ArenaLayout l = arena_layout(cfg);
+    if (cfg->arena_bytes < l.total) return EVK_ERR_WORKSPACE;
+    evk_mem *m = new (std::nothrow) evk_mem;
+    if (!m) return EVK_ERR_INVALID;
+    m->cfg = *cfg;
+    m->size = 0;
+    char *base = static_cast<char *>(cfg->arena);
+    m->bank = reinterpret_cast<__nv_bfloat16 *>(base + l.bank);
+    m->q_tables = reinterpret_cast<float *>(base + l.q_tables);
+    m->status = reinterpret_cast<int32_t *>(base + l.status);
+    m->scoring = EVK_SCORING_AUTO;
+    m->launches = 0;
+    cudaError_t err = cudaMemsetAsync(m->status, 0, 256, 0);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(0);
+    if (err != cudaSuccess) {
+        delete m;
+        return EVK_ERR_CUDA;
+    }
+    *out = m;
+    return EVK_OK;
+}
+
+int evk_mem_destroy(evk_mem *mem) {
+    delete mem;
+    return EVK_OK;
+}
+
+int64_t evk_mem_size(const evk_mem *mem) { return mem ? mem->size : 0; }
+
+int64_t evk_launch_count(const evk_mem *mem) { return mem ? mem->launches : 0; }
+
+int evk_mem_set_scoring(evk_mem *mem, int mode) {
+    if (!mem || mode < EVK_SCORING_AUTO || mode > EVK_SCORING_TENSOR) return EVK_ERR_INVALID;
+    mem->scoring = mode;
+    return EVK_OK;
+}
+
+int evk_mem_insert(evk_mem *mem, const void *emb, int emb_dtype, int64_t n, int stage,
+                   const float *q_init, int32_t *ids_out, void *stream) {
+    if (!mem || n < 0 || (emb_dtype != EVK_DTYPE_F32 && emb_dtype != EVK_DTYPE_BF16)) return EVK_ERR_INVALID;
+    if (stage != EVK_STAGE_ALL && !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!emb || !aligned(emb, 16)) return EVK_ERR_INVALID;
+    if (mem->size + n > mem->cfg.capacity) return EVK_ERR_CAPACITY;
+    int launches = 0;
+    cudaError_t err = launch_insert(mem->bank, mem->q_tables, mem->status, mem->cfg.capacity, mem->cfg.d,
+                                    mem->cfg.n_stages, mem->size, n, emb, emb_dtype, stage, q_init,
+                                    mem->cfg.q_default, ids_out, static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    if (err != cudaSuccess) return EVK_ERR_CUDA;
+    mem->size += n;
+    return EVK_OK;
+}
+
+size_t evk_retrieve_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1) {
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1) return 0;
+    return retrieve_layout(mem, B, k1).total + 256;
+}
+
+int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage,
+                 int32_t k1, int32_t k2, float w,
+                 int32_t *ids_out, float *scores_out,
+                 int32_t *pool_ids_out, float *pool_sims_out,
+                 void *workspace, size_t workspace_bytes, void *stream_v) {
+    if (!mem || B < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return EVK_ERR_INVALID;
+    if (!(w >= 0.0f && w <= 1.0f)) return EVK_ERR_INVALID;
+    if (q_dtype != EVK_DTYPE_F32 && q_dtype != EVK_DTYPE_BF16) return EVK_ERR_INVALID;
+    if (B == 0) return EVK_OK;
+    if (!queries || !aligned(queries, 16) || !ids_out || !scores_out) return EVK_ERR_INVALID;
+    if (!workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    const RetrieveLayout l = retrieve_layout(mem, B, k1);
+    if (workspace_bytes < l.total) return EVK_ERR_WORKSPACE;
+    if (mem->scoring == EVK_SCORING_TENSOR) return EVK_ERR_UNSUPPORTED;
+    if (!stream_supported(mem->cfg.d)) return EVK_ERR_UNSUPPORTED;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    char *ws = static_cast<char *>(workspace);
+    int launches = 0;
+    cudaError_t err = cudaSuccess;
+
+    const __nv_bfloat16 *q_bf16 = static_cast<const __nv_bfloat16 *>(queries);
+    if (q_dtype == EVK_DTYPE_F32) {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(ws + l.q_bf16);
+        err = launch_convert_queries(static_cast<const float *>(queries), dst, (int64_t)B * mem->cfg.d, stream, &launches);
+        q_bf16 = dst;
+    }
+
+    int32_t *pool_ids = reinterpret_cast<int32_t *>(ws + l.pool_ids);
+    float *pool_sims = reinterpret_cast<float *>(ws + l.pool_sims);
+    int *part_counts = reinterpret_cast<int *>(ws + l.part_counts);
+    uint64_t *part_keys = reinterpret_cast<uint64_t *>(ws + l.part_keys);
+
+    int nparts = 0;
+    if (err == cudaSuccess && mem->size > 0) {
+        const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+        nparts = plan.nparts;
+        err = launch_score_stream(mem->bank, mem->size, mem->cfg.d, q_bf16, B, k1, plan, part_keys,
+                                  part_counts, stream, &launches);
+    }
+    if (err == cudaSuccess)
+        err = launch_merge_pool(part_keys, part_counts, nparts, k1, B, k1, pool_ids, pool_sims,
+                                pool_ids_out, pool_sims_out, stream, &launches);
+    if (err == cudaSuccess)
+        err = launch_rerank(pool_ids, pool_sims, B, k1, k2, mem->q_tables + (size_t)stage * mem->cfg.capacity,
+                            w, ids_out, scores_out, stream, &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+size_t evk_q_update_workspace_bytes(const evk_mem *mem, int64_t M) {
+    if (!mem || M < 0) return 0;
+    return q_update_workspace_bytes(M) + 256;
+}
+
+int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
+                 const float *rewards, float alpha,
+                 void *workspace, size_t workspace_bytes, void *stream) {
+    if (!mem || M < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (!(alpha > 0.0f && alpha <= 1.0f)) return EVK_ERR_INVALID;
+    if (M == 0) return EVK_OK;
+    if (M >= ((int64_t)1 << 31)) return EVK_ERR_UNSUPPORTED;
+    if (!ids || !rewards || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (workspace_bytes < q_update_workspace_bytes(M)) return EVK_ERR_WORKSPACE;
+    int launches = 0;
+    cudaError_t err = launch_q_update(mem->q_tables + (size_t)stage * mem->cfg.capacity, mem->size, ids, rewards,
+                                      M, alpha, mem->status, workspace, static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream) {
+    if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!out) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemcpyAsync(out, mem->q_tables + (size_t)stage * mem->cfg.capacity + first,
+                                       (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+int evk_q_write(evk_mem *mem, int stage, int64_t first, int64_t n, const float *values, void *stream) {
+    if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!values) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemcpyAsync(mem->q_tables + (size_t)stage * mem->cfg.capacity + first, values,
+                                       (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+int evk_bank_read(evk_mem *mem, int64_t first, int64_t n, void *out_bf16, void *stream) {
+    if (!mem || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!out_bf16) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemcpyAsync(out_bf16, mem->bank + (size_t)first * mem->cfg.d,
+                                       (size_t)n * mem->cfg.d * sizeof(__nv_bfloat16), cudaMemcpyDeviceToDevice,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+// ---- host-buffer forms -------------------------------------------------------
+
+size_t evk_retrieve_host_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1, int32_t k2) {
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return 0;
+    const size_t b = (size_t)B;
+    return align256(b * mem->cfg.d * sizeof(float)) + 2 * align256(b * k2 * sizeof(float)) +
+           evk_retrieve_workspace_bytes(mem, B, k1);
+}
+
+int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32_t B, int stage,
+                      int32_t k1, int32_t k2, float w,
+                      int32_t *ids_out_host, float *scores_out_host,
+                      void *workspace, size_t workspace_bytes, void *stream_v) {
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return EVK_ERR_INVALID;
+    if (q_dtype != EVK_DTYPE_F32 && q_dtype != EVK_DTYPE_BF16) return EVK_ERR_INVALID;
+    if (B == 0) return EVK_OK;
+    if (!queries_host || !ids_out_host || !scores_out_host || !workspace || !aligned(workspace, 256))
+        return EVK_ERR_INVALID;
+    if (workspace_bytes < evk_retrieve_host_workspace_bytes(mem, B, k1, k2)) return EVK_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t b = (size_t)B;
+    const size_t q_bytes = b * mem->cfg.d * (q_dtype == EVK_DTYPE_F32 ? sizeof(float) : sizeof(__nv_bfloat16));
+    char *ws = static_cast<char *>(workspace);
+    void *q_dev = ws;
+    int32_t *ids_dev = reinterpret_cast<int32_t *>(ws + align256(b * mem->cfg.d * sizeof(float)));
+    float *scores_dev = reinterpret_cast<float *>(reinterpret_cast<char *>(ids_dev) + align256(b * k2 * sizeof(float)));
+    char *inner = reinterpret_cast<char *>(scores_dev) + align256(b * k2 * sizeof(float));
+    const size_t inner_bytes = workspace_bytes - (size_t)(inner - ws);
+    if (cudaMemcpyAsync(q_dev, queries_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return EVK_ERR_CUDA;
+    int rc = evk_retrieve(mem, q_dev, q_dtype, B, stage, k1, k2, w, ids_dev, scores_dev, nullptr, nullptr,
+                          inner, inner_bytes, stream_v);
+    if (rc != EVK_OK) return rc;
+    if (cudaMemcpyAsync(ids_out_host, ids_dev, b * k2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(scores_out_host, scores_dev, b * k2 * sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return EVK_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(stream));
+}
+
+size_t evk_q_update_host_workspace_bytes(const evk_mem *mem, int64_t M) {
+    if (!mem || M < 0) return 0;
+    return 2 * align256((size_t)M * 4) + evk_q_update_workspace_bytes(mem, M);
+}
+
+int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stage,
+                      const float *rewards_host, float alpha,
+                      void *workspace, size_t workspace_bytes, void *stream_v) {
+    if (!mem || M < 0) return EVK_ERR_INVALID;
+    if (M == 0) return EVK_OK;
+    if (!ids_host || !rewards_host || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (workspace_bytes < evk_q_update_host_workspace_bytes(mem, M)) return EVK_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    char *ws = static_cast<char *>(workspace);
+    int32_t *ids_dev = reinterpret_cast<int32_t *>(ws);
+    float *r_dev = reinterpret_cast<float *>(ws + align256((size_t)M * 4));
+    char *inner = ws + 2 * align256((size_t)M * 4);
+    if (cudaMemcpyAsync(ids_dev, ids_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(r_dev, rewards_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return EVK_ERR_CUDA;
+    int rc = evk_q_update(mem, ids_dev, M, stage, r_dev, alpha, inner, workspace_bytes - (size_t)(inner - ws), stream_v);
+    if (rc != EVK_OK) return rc;
+    return cuda_status(cudaStreamSynchronize(stream));
+}
+
+int evk_last_status(evk_mem *mem, void *stream_v) {
+    if (!mem) return EVK_ERR_INVALID;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, mem->status, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return EVK_ERR_CUDA;
+    if (cudaMemsetAsync(mem->status, 0, sizeof(word), stream) != cudaSuccess) return EVK_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return EVK_ERR_CUDA;
+    return word;
+}
+
+const char *evk_strerror(int status) {
+    switch (status) {
+        case EVK_OK: return "ok";
+        case EVK_ERR_INVALID: return "invalid argument";
+        case EVK_ERR_CAPACITY: return "bank capacity exceeded";
+        case EVK_ERR_WORKSPACE: return "workspace or arena too small";
+        case EVK_ERR_RANGE: return "entry id out of range";
+        case EVK_ERR_NONFINITE: return "non-finite reward";
+        case EVK_ERR_DEVICE_TIMEOUT: return "bounded wait in a kernel ran out";
+        case EVK_ERR_CUDA: return "CUDA call failed";
+        case EVK_ERR_UNSUPPORTED: return "unsupported shape";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

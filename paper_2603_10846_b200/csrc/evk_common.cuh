@@ -1,0 +1,129 @@
+// Shared device helpers: ranking keys, block-wide selection, launch plumbing.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "evk.h"
+
+namespace evk {
+
+constexpr int kNumSM = 148;            // B200: 2 dies x 74 SMs
+constexpr uint32_t kPadId = 0xffffffffu;
+
+// ---------------------------------------------------------------------------
+// Ranking keys.  A candidate (sim, id) is packed into one 64-bit integer so that
+// "larger key" means "ranks earlier": similarity descending, then id ascending.
+// The float is mapped to an unsigned integer with the same order; the id is
+// stored complemented.  Keys of distinct entries are distinct.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t ordered_bits(float f) {
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t o) {
+    uint32_t u = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+    return __uint_as_float(u);
+}
+__device__ __forceinline__ uint64_t make_key(float sim, int32_t id) {
+    sim += 0.0f;  // -0 -> +0: equal similarities must tie exactly
+    return ((uint64_t)ordered_bits(sim) << 32) | (uint32_t)(~(uint32_t)id);
+}
+__device__ __forceinline__ float key_sim(uint64_t key) { return from_ordered_bits((uint32_t)(key >> 32)); }
+__device__ __forceinline__ int32_t key_id(uint64_t key) { return (int32_t)(~(uint32_t)key); }
+
+// ---------------------------------------------------------------------------
+// Block-wide exact selection.  Keeps the k largest of n distinct 64-bit keys held
+// in shared memory and moves them to keys[0..k) (in no particular order).
+// Most-significant-digit radix select, 8 bits per pass, followed by an in-place
+// compaction through registers.  Every thread of the block must call it with the
+// same arguments; n <= NT * PER_THREAD; 0 < k < n.  Returns the k-th largest key.
+//   hist: 256 ints of shared memory; scal: 4 uint64 of shared memory.
+// ---------------------------------------------------------------------------
+template <int NT, int PER_THREAD>
+__device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, uint64_t *scal) {
+    const int tid = threadIdx.x;
+    uint64_t prefix = 0, mask = 0;
+    int kk = k;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += NT) hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += NT) {
+            uint64_t key = keys[i];
+            if ((key & mask) == prefix) atomicAdd(&hist[(int)((key >> shift) & 0xff)], 1);
+        }
+        __syncthreads();
+        if (tid < 32) {
+            // lane l owns bins [8l, 8l+8); find the bin holding the kk-th largest, from the top.
+            int local[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { local[j] = hist[tid * 8 + j]; sum += local[j]; }
+            int incl = sum;  // becomes the total of this lane and every higher lane
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                int v = __shfl_down_sync(0xffffffffu, incl, off);
+                if (tid + off < 32) incl += v;
+            }
+            const int above = incl - sum;
+            if (above < kk && kk <= above + sum) {  // exactly one lane
+                int c = above, digit = tid * 8;
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    if (kk <= c + local[j]) { digit = tid * 8 + j; break; }
+                    c += local[j];
+                }
+                scal[0] = prefix | ((uint64_t)digit << shift);
+                scal[1] = (uint64_t)(kk - c);
+            }
+        }
+        __syncthreads();
+        prefix = scal[0];
+        kk = (int)scal[1];
+        mask |= (uint64_t)0xff << shift;
+        __syncthreads();
+    }
+    // prefix is now the k-th largest key; exactly k keys are >= prefix.
+    uint64_t mine[PER_THREAD];
+#pragma unroll
+    for (int j = 0; j < PER_THREAD; ++j) {
+        int i = tid + j * NT;
+        mine[j] = (i < n) ? keys[i] : 0;
+    }
+    int *counter = reinterpret_cast<int *>(&scal[2]);
+    if (tid == 0) *counter = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < PER_THREAD; ++j) {
+        int i = tid + j * NT;
+        if (i < n && mine[j] >= prefix) keys[atomicAdd(counter, 1)] = mine[j];
+    }
+    __syncthreads();
+    return prefix;
+}
+
+// Block-wide bitonic sort of n_pow2 keys in shared memory, descending.
+template <int NT>
+__device__ void block_sort_desc(uint64_t *keys, int n_pow2) {
+    for (int size = 2; size <= n_pow2; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int t = threadIdx.x; t < (n_pow2 >> 1); t += NT) {
+                int lo = 2 * t - (t & (stride - 1));
+                int hi = lo + stride;
+                bool desc = ((lo & size) == 0);
+                uint64_t a = keys[lo], b = keys[hi];
+                if ((a < b) == desc) { keys[lo] = b; keys[hi] = a; }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+__host__ __device__ __forceinline__ int next_pow2(int x) {
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+}  // namespace evk

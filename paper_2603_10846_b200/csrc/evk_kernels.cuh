@@ -1,0 +1,54 @@
+// Host-side launchers of the kernels, one per step of the hot path.  Each returns a
+// cudaError_t from the launch; none synchronises.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace evk {
+
+// ---- insert (Eq. 1) ---------------------------------------------------------
+cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, int32_t *status, int64_t capacity,
+                          int d, int n_stages, int64_t first, int64_t n, const void *emb, int emb_dtype,
+                          int stage, const float *q_init, float q_default, int32_t *ids_out,
+                          cudaStream_t stream, int *launches);
+
+// fp32 -> bf16 (nearest even) conversion of a query batch.
+cudaError_t launch_convert_queries(const float *src, __nv_bfloat16 *dst, int64_t n_elems,
+                                   cudaStream_t stream, int *launches);
+
+// ---- phase 1, streaming kernel ---------------------------------------------
+// Candidate lists: for query q and part p, part_counts[q*nparts+p] keys at
+// part_keys[(q*nparts+p)*part_stride ...].
+struct StreamPlan {
+    int qb;        // queries per pass over the bank
+    int nparts;    // thread blocks per pass (= candidate lists per query)
+    int cap;       // shared-memory candidate capacity per query
+    size_t smem;   // dynamic shared memory per block
+};
+bool stream_supported(int d);
+StreamPlan stream_plan(int64_t size, int d, int B, int k1);
+cudaError_t launch_score_stream(const __nv_bfloat16 *bank, int64_t size, int d,
+                                const __nv_bfloat16 *queries, int B, int k1, const StreamPlan &plan,
+                                uint64_t *part_keys, int *part_counts, cudaStream_t stream, int *launches);
+
+// ---- phase 1, pool merge ----------------------------------------------------
+constexpr int kMergeMaxParts = 2048;
+cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
+                              int part_stride, int B, int k1, int32_t *pool_ids, float *pool_sims,
+                              int32_t *pool_ids_user, float *pool_sims_user,
+                              cudaStream_t stream, int *launches);
+
+// ---- phase 2, rerank --------------------------------------------------------
+cudaError_t launch_rerank(const int32_t *pool_ids, const float *pool_sims, int B, int k1, int k2,
+                          const float *q_stage, float w, int32_t *ids_out, float *scores_out,
+                          cudaStream_t stream, int *launches);
+
+// ---- Eq. 4 update -----------------------------------------------------------
+size_t q_update_workspace_bytes(int64_t m);
+cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
+                            int64_t m, float alpha, int32_t *status, void *workspace,
+                            cudaStream_t stream, int *launches);
+
+}  // namespace evk

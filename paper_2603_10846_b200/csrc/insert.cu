@@ -1,0 +1,81 @@
+// Appending experiences to the memory (Eq. 1): embeddings become bf16 rows of the
+// bank, and each new entry gets one value estimate per stage.
+#include "evk_common.cuh"
+#include "evk_kernels.cuh"
+
+namespace evk {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// 8 elements per thread: two 16-byte loads of fp32 (or one of bf16), one 16-byte store.
+__global__ void __launch_bounds__(kThreads)
+insert_rows_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int is_bf16, int64_t n_vec) {
+    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * kThreads) {
+        uint4 out;
+        if (is_bf16) {
+            out = reinterpret_cast<const uint4 *>(src)[i];
+        } else {
+            const float4 a = reinterpret_cast<const float4 *>(src)[2 * i];
+            const float4 b = reinterpret_cast<const float4 *>(src)[2 * i + 1];
+            __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y);
+            __nv_bfloat162 p1 = __floats2bfloat162_rn(a.z, a.w);
+            __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y);
+            __nv_bfloat162 p3 = __floats2bfloat162_rn(b.z, b.w);
+            out.x = *reinterpret_cast<uint32_t *>(&p0);
+            out.y = *reinterpret_cast<uint32_t *>(&p1);
+            out.z = *reinterpret_cast<uint32_t *>(&p2);
+            out.w = *reinterpret_cast<uint32_t *>(&p3);
+        }
+        reinterpret_cast<uint4 *>(dst)[i] = out;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+insert_values_kernel(float *__restrict__ q_tables, int64_t capacity, int n_stages, int64_t first, int64_t n,
+                     int stage, const float *__restrict__ q_init, float q_default, int32_t *__restrict__ ids_out) {
+    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kThreads) {
+        const float v = q_init ? q_init[i] : q_default;
+        for (int s = 0; s < n_stages; ++s)
+            q_tables[(int64_t)s * capacity + first + i] = (stage < 0 || s == stage) ? v : q_default;
+        if (ids_out) ids_out[i] = (int32_t)(first + i);
+    }
+}
+
+int grid_for(int64_t work_items) {
+    int64_t g = (work_items + kThreads - 1) / kThreads;
+    const int64_t cap = (int64_t)kNumSM * 8;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+}  // namespace
+
+cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, int32_t *status, int64_t capacity,
+                          int d, int n_stages, int64_t first, int64_t n, const void *emb, int emb_dtype,
+                          int stage, const float *q_init, float q_default, int32_t *ids_out,
+                          cudaStream_t stream, int *launches) {
+    (void)status;
+    if (n <= 0) return cudaSuccess;
+    const int64_t n_vec = n * d / 8;
+    insert_rows_kernel<<<grid_for(n_vec), kThreads, 0, stream>>>(bank + first * d, emb, emb_dtype == EVK_DTYPE_BF16, n_vec);
+    ++*launches;
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    insert_values_kernel<<<grid_for(n), kThreads, 0, stream>>>(q_tables, capacity, n_stages, first, n, stage, q_init, q_default, ids_out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_convert_queries(const float *src, __nv_bfloat16 *dst, int64_t n_elems,
+                                   cudaStream_t stream, int *launches) {
+    if (n_elems <= 0) return cudaSuccess;
+    const int64_t n_vec = n_elems / 8;
+    insert_rows_kernel<<<grid_for(n_vec), kThreads, 0, stream>>>(dst, src, 0, n_vec);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace evk

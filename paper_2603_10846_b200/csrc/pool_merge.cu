@@ -1,0 +1,129 @@
+// Phase 1, last step: merge the candidate lists that the scoring kernels left per
+// (query, part) into the final pool C(x) of Section 3.2 — the k1 entries of largest
+// similarity, written in (similarity descending, id ascending) order.
+//
+// One thread block per query.  Candidates stream through a shared-memory buffer
+// that is cut back to its best k1 by an exact radix select whenever it fills; the
+// survivors are then sorted with a bitonic network.  Because keys are totally
+// ordered and distinct, the result does not depend on the order in which the
+// scoring kernels appended candidates.
+#include "evk_common.cuh"
+#include "evk_kernels.cuh"
+
+namespace evk {
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kSelPerThread = 8;
+constexpr int kCap = kThreads * kSelPerThread;  // 4096 keys = 32 KB
+constexpr int kBatch = 2048;                    // candidates examined between capacity checks
+
+__global__ void __launch_bounds__(kThreads)
+merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
+                  int part_stride, int k1, int32_t *__restrict__ pool_ids, float *__restrict__ pool_sims,
+                  int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user) {
+    __shared__ __align__(16) uint64_t keys[kCap];
+    __shared__ int offs[kMergeMaxParts + 1];
+    __shared__ int hist[256];
+    __shared__ uint64_t scal[4];
+    __shared__ int count;
+    __shared__ uint64_t tau;
+
+    const int tid = threadIdx.x;
+    const int q = blockIdx.x;
+    const int *cnt = part_counts + (size_t)q * nparts;
+
+    // exclusive scan of the part counts (single thread per 8 parts, then serial over chunks:
+    // nparts is at most a few thousand)
+    if (tid == 0) {
+        count = 0;
+        tau = 0;
+    }
+    for (int p = tid; p < nparts; p += kThreads) offs[p + 1] = cnt[p];
+    if (tid == 0) offs[0] = 0;
+    __syncthreads();
+    if (tid < 32) {
+        // warp-serial inclusive scan in chunks of 32
+        int carry = 0;
+        for (int base = 0; base < nparts; base += 32) {
+            int p = base + tid;
+            int v = (p < nparts) ? offs[p + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                int u = __shfl_up_sync(0xffffffffu, v, off);
+                if (tid >= off) v += u;
+            }
+            if (p < nparts) offs[p + 1] = v + carry;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+    const int total = offs[nparts];
+
+    for (int base = 0; base < total; base += kBatch) {
+        const uint64_t t = tau;
+#pragma unroll
+        for (int j = 0; j < kBatch / kThreads; ++j) {
+            const int idx = base + tid + j * kThreads;
+            if (idx < total) {
+                // part p with offs[p] <= idx < offs[p+1]
+                int lo = 0, hi = nparts;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (offs[mid] <= idx) lo = mid; else hi = mid;
+                }
+                const uint64_t key = part_keys[((size_t)q * nparts + lo) * part_stride + (idx - offs[lo])];
+                if (key > t) keys[atomicAdd(&count, 1)] = key;
+            }
+        }
+        __syncthreads();
+        const int n = count;
+        if (n > kCap - kBatch && n > k1) {
+            const uint64_t kth = block_select_topk<kThreads, kSelPerThread>(keys, n, k1, hist, scal);
+            if (tid == 0) {
+                count = k1;
+                tau = kth;
+            }
+        }
+        __syncthreads();
+    }
+
+    int n = count;
+    if (n > k1) {
+        block_select_topk<kThreads, kSelPerThread>(keys, n, k1, hist, scal);
+        n = k1;
+    }
+    const int np2 = next_pow2(n > 1 ? n : 1);
+    for (int i = n + tid; i < np2; i += kThreads) keys[i] = 0;
+    __syncthreads();
+    block_sort_desc<kThreads>(keys, np2);
+    for (int i = tid; i < k1; i += kThreads) {
+        int32_t id = -1;
+        float s = -INFINITY;
+        if (i < n) {
+            id = key_id(keys[i]);
+            s = key_sim(keys[i]);
+        }
+        pool_ids[(size_t)q * k1 + i] = id;
+        pool_sims[(size_t)q * k1 + i] = s;
+        if (pool_ids_user) pool_ids_user[(size_t)q * k1 + i] = id;
+        if (pool_sims_user) pool_sims_user[(size_t)q * k1 + i] = s;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
+                              int part_stride, int B, int k1, int32_t *pool_ids, float *pool_sims,
+                              int32_t *pool_ids_user, float *pool_sims_user,
+                              cudaStream_t stream, int *launches) {
+    if (B <= 0) return cudaSuccess;
+    if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
+    merge_pool_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, k1,
+                                                  pool_ids, pool_sims, pool_ids_user, pool_sims_user);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace evk

@@ -1,0 +1,256 @@
+// The unified value update (Eq. 4; Eq. 8 in Appendix A):
+//
+//   Q_stage[id] <- Q + alpha * (r - Q)        for each (id, r) of the batch, in array order.
+//
+// An id may occur many times in one batch (popular entries are retrieved often),
+// and binary32 arithmetic is not associative, so the stored bits depend on the
+// order in which one entry's rewards are applied.  The order is fixed to array
+// order: the batch is sorted by id with a STABLE radix sort (so each entry's
+// rewards stay in array order), and one thread then walks each entry's run of
+// rewards sequentially with three separately rounded operations.  Entries with
+// different ids do not interact, so they run in parallel.
+//
+// A checking pass runs first; if any id is out of range or any reward is not
+// finite, nothing is written and the status word records why.
+#include "evk_common.cuh"
+#include "evk_kernels.cuh"
+
+namespace evk {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kPerThread = 8;
+constexpr int kTile = kThreads * kPerThread;  // 2048 elements per block and pass
+
+constexpr int kFlagRange = 1, kFlagNonFinite = 2;
+
+__global__ void __launch_bounds__(kThreads)
+validate_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int64_t m, int64_t size,
+                int *__restrict__ flags) {
+    int bad = 0;
+    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < m; i += (int64_t)gridDim.x * kThreads) {
+        const int32_t id = ids[i];
+        if (id < 0 || id >= size) bad |= kFlagRange;
+        const float r = rewards[i];
+        if (!(fabsf(r) <= 3.402823466e38f)) bad |= kFlagNonFinite;
+    }
+    bad = __reduce_or_sync(0xffffffffu, bad);
+    if ((threadIdx.x & 31) == 0 && bad) atomicOr(flags, bad);
+}
+
+// Per-block histogram of one 8-bit digit; hist is digit-major: hist[digit * nb + block].
+__global__ void __launch_bounds__(kThreads)
+radix_hist_kernel(const int32_t *__restrict__ keys, int64_t m, int shift, int nb, const int *__restrict__ flags,
+                  int *__restrict__ hist) {
+    if (*flags) return;
+    __shared__ int h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kTile;
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const int64_t e = base + threadIdx.x + j * kThreads;
+        if (e < m) atomicAdd(&h[(keys[e] >> shift) & 0xff], 1);
+    }
+    __syncthreads();
+    hist[threadIdx.x * nb + blockIdx.x] = h[threadIdx.x];
+}
+
+// Exclusive scan of n ints in place, one block.
+__global__ void __launch_bounds__(1024)
+scan_kernel(int *__restrict__ data, int n, const int *__restrict__ flags) {
+    if (*flags) return;
+    __shared__ int warp_sums[32];
+    __shared__ int carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int base = 0; base < n; base += 1024) {
+        const int i = base + tid;
+        const int v = (i < n) ? data[i] : 0;
+        int x = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, x, off);
+            if (lane >= off) x += u;
+        }
+        if (lane == 31) warp_sums[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int s = warp_sums[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, s, off);
+                if (lane >= off) s += u;
+            }
+            warp_sums[lane] = s;  // inclusive over warps
+        }
+        __syncthreads();
+        const int carry = carry_s;
+        const int before = (warp ? warp_sums[warp - 1] : 0) + carry;
+        if (i < n) data[i] = before + x - v;
+        __syncthreads();
+        if (tid == 1023) carry_s = before + x;
+        __syncthreads();
+    }
+}
+
+// Stable scatter of one digit.  Warp w owns the 256 consecutive elements
+// [tile + 256w, tile + 256w + 256) and visits them 32 at a time in order, so ranks
+// within a digit follow array order inside the warp, warps are ordered by prefix
+// sums, and blocks by the scanned histogram.
+__global__ void __launch_bounds__(kThreads)
+radix_scatter_kernel(const int32_t *__restrict__ keys_in, const float *__restrict__ vals_in, int64_t m,
+                     int shift, int nb, const int *__restrict__ flags, const int *__restrict__ offsets,
+                     int32_t *__restrict__ keys_out, float *__restrict__ vals_out) {
+    if (*flags) return;
+    __shared__ int warp_cnt[kWarps][256];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < kWarps * 256; i += kThreads) (&warp_cnt[0][0])[i] = 0;
+    __syncthreads();
+
+    const int64_t base = (int64_t)blockIdx.x * kTile + warp * (32 * kPerThread);
+    int32_t key[kPerThread];
+    float val[kPerThread];
+    int rank[kPerThread];
+    const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+    for (int r = 0; r < kPerThread; ++r) {
+        const int64_t e = base + r * 32 + lane;
+        const bool valid = e < m;
+        key[r] = valid ? keys_in[e] : 0;
+        val[r] = valid ? vals_in[e] : 0.0f;
+        const int digit = valid ? ((key[r] >> shift) & 0xff) : 256;
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        int old = 0;
+        if (valid) old = warp_cnt[warp][digit];
+        __syncwarp();
+        if (valid && (peers & lt_mask) == 0) warp_cnt[warp][digit] = old + __popc(peers);
+        __syncwarp();
+        rank[r] = old + __popc(peers & lt_mask);
+    }
+    __syncthreads();
+    {
+        // digit `tid`: turn per-warp counts into starting offsets
+        int run = offsets[tid * nb + blockIdx.x];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const int t = warp_cnt[w][tid];
+            warp_cnt[w][tid] = run;
+            run += t;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kPerThread; ++r) {
+        const int64_t e = base + r * 32 + lane;
+        if (e < m) {
+            const int digit = (key[r] >> shift) & 0xff;
+            const int dst = warp_cnt[warp][digit] + rank[r];
+            keys_out[dst] = key[r];
+            vals_out[dst] = val[r];
+        }
+    }
+}
+
+// One thread per run of equal ids (the thread at the run's first element).
+__global__ void __launch_bounds__(kThreads)
+apply_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int64_t m, float alpha,
+             float *__restrict__ q_stage, const int *__restrict__ flags, int32_t *__restrict__ status) {
+    const int f = *flags;
+    if (f) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && *status == 0)
+            *status = (f & kFlagRange) ? EVK_ERR_RANGE : EVK_ERR_NONFINITE;
+        return;
+    }
+    const int64_t t = blockIdx.x * (int64_t)kThreads + threadIdx.x;
+    if (t >= m) return;
+    const int32_t id = ids[t];
+    if (t > 0 && ids[t - 1] == id) return;
+    // end of the run: first index > t whose id differs (ids are sorted)
+    int64_t end = t + 1;
+    if (end < m && ids[end] == id) {
+        int64_t lo = end, hi = m;  // ids[lo] == id, ids[hi] != id (or hi == m)
+        while (hi - lo > 1) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (ids[mid] == id) lo = mid; else hi = mid;
+        }
+        end = hi;
+    }
+    float q = q_stage[id];
+    for (int64_t j = t; j < end; ++j) {
+        const float diff = __fsub_rn(rewards[j], q);
+        const float step = __fmul_rn(alpha, diff);
+        q = __fadd_rn(q, step);
+    }
+    q_stage[id] = q;
+}
+
+int num_blocks(int64_t m) { return (int)((m + kTile - 1) / kTile); }
+
+struct UpdateLayout {
+    size_t flags, hist, keys_a, vals_a, keys_b, vals_b, total;
+};
+
+UpdateLayout layout_for(int64_t m) {
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    UpdateLayout l;
+    const size_t nb = (size_t)num_blocks(m > 0 ? m : 1);
+    l.flags = 0;
+    l.hist = 256;
+    l.keys_a = l.hist + align(256 * nb * sizeof(int));
+    l.vals_a = l.keys_a + align((size_t)m * 4);
+    l.keys_b = l.vals_a + align((size_t)m * 4);
+    l.vals_b = l.keys_b + align((size_t)m * 4);
+    l.total = l.vals_b + align((size_t)m * 4);
+    return l;
+}
+
+}  // namespace
+
+size_t q_update_workspace_bytes(int64_t m) { return layout_for(m).total; }
+
+cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
+                            int64_t m, float alpha, int32_t *status, void *workspace,
+                            cudaStream_t stream, int *launches) {
+    if (m <= 0) return cudaSuccess;
+    const UpdateLayout l = layout_for(m);
+    char *ws = static_cast<char *>(workspace);
+    int *flags = reinterpret_cast<int *>(ws + l.flags);
+    int *hist = reinterpret_cast<int *>(ws + l.hist);
+    int32_t *keys[2] = {reinterpret_cast<int32_t *>(ws + l.keys_a), reinterpret_cast<int32_t *>(ws + l.keys_b)};
+    float *vals[2] = {reinterpret_cast<float *>(ws + l.vals_a), reinterpret_cast<float *>(ws + l.vals_b)};
+    const int nb = num_blocks(m);
+
+    cudaError_t err = cudaMemsetAsync(flags, 0, sizeof(int), stream);
+    if (err != cudaSuccess) return err;
+    int vgrid = (int)((m + kThreads - 1) / kThreads);
+    if (vgrid > kNumSM * 8) vgrid = kNumSM * 8;
+    validate_kernel<<<vgrid, kThreads, 0, stream>>>(ids, rewards, m, size, flags);
+    ++*launches;
+
+    int bits = 0;
+    while (bits < 31 && ((int64_t)1 << bits) < size) ++bits;
+    int passes = (bits + 7) / 8;
+    if (passes < 1) passes = 1;
+
+    const int32_t *k_in = ids;
+    const float *v_in = rewards;
+    for (int p = 0; p < passes; ++p) {
+        int32_t *k_out = keys[p & 1];
+        float *v_out = vals[p & 1];
+        radix_hist_kernel<<<nb, kThreads, 0, stream>>>(k_in, m, 8 * p, nb, flags, hist);
+        scan_kernel<<<1, 1024, 0, stream>>>(hist, 256 * nb, flags);
+        radix_scatter_kernel<<<nb, kThreads, 0, stream>>>(k_in, v_in, m, 8 * p, nb, flags, hist, k_out, v_out);
+        *launches += 3;
+        k_in = k_out;
+        v_in = v_out;
+    }
+    apply_kernel<<<(int)((m + kThreads - 1) / kThreads), kThreads, 0, stream>>>(k_in, v_in, m, alpha, q_stage, flags, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace evk

@@ -1,0 +1,305 @@
+"""Python binding of the C-ABI library ``libevk.so`` (see ``include/evk.h``).
+
+Argument marshalling only: tensors are checked for device, dtype and contiguity
+and handed to the library as raw pointers; every step of retrieval and of the
+value update runs in the library's CUDA kernels.  PyTorch supplies device memory
+and streams.  There is no CPU fallback: importing this module without the built
+library raises, and calling into it without a CUDA device fails in the library.
+
+Function names mirror the C ABI: ``evk_mem_create``, ``evk_mem_insert``,
+``evk_retrieve``, ``evk_q_update`` and the helpers around them.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libevk.so")
+
+EVK_OK = 0
+EVK_ERR_INVALID = -1
+EVK_ERR_CAPACITY = -2
+EVK_ERR_WORKSPACE = -3
+EVK_ERR_RANGE = -4
+EVK_ERR_NONFINITE = -5
+EVK_ERR_DEVICE_TIMEOUT = -6
+EVK_ERR_CUDA = -7
+EVK_ERR_UNSUPPORTED = -8
+
+EVK_DTYPE_F32, EVK_DTYPE_BF16 = 0, 1
+EVK_STAGE_DRAFT, EVK_STAGE_REFINE, EVK_STAGE_ALL = 0, 1, -1
+EVK_SCORING_AUTO, EVK_SCORING_STREAM, EVK_SCORING_TENSOR = 0, 1, 2
+EVK_MAX_K1 = 1024
+
+# Every symbol include/evk.h declares.
+EXPORTS = (
+    "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
+    "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
+    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_read", "evk_q_write", "evk_bank_read",
+    "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
+    "evk_q_update_host", "evk_last_status", "evk_launch_count", "evk_strerror",
+)
+
+
+class EvkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("n_stages", ctypes.c_int32), ("capacity", ctypes.c_int64),
+                ("q_default", ctypes.c_float), ("reserved", ctypes.c_int32),
+                ("arena", ctypes.c_void_p), ("arena_bytes", ctypes.c_size_t)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2603_10846_b200.build` "
+            "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+    cint = ctypes.c_int
+    cfgp = ctypes.POINTER(_Config)
+    sig = {
+        "evk_mem_bytes_required": (sz, [cfgp]),
+        "evk_mem_create": (cint, [cfgp, ctypes.POINTER(vp)]),
+        "evk_mem_destroy": (cint, [vp]),
+        "evk_mem_size": (i64, [vp]),
+        "evk_mem_set_scoring": (cint, [vp, cint]),
+        "evk_mem_insert": (cint, [vp, vp, cint, i64, cint, vp, vp, vp]),
+        "evk_retrieve_workspace_bytes": (sz, [vp, i32, i32]),
+        "evk_retrieve": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]),
+        "evk_q_update_workspace_bytes": (sz, [vp, i64]),
+        "evk_q_update": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
+        "evk_q_read": (cint, [vp, cint, i64, i64, vp, vp]),
+        "evk_q_write": (cint, [vp, cint, i64, i64, vp, vp]),
+        "evk_bank_read": (cint, [vp, i64, i64, vp, vp]),
+        "evk_retrieve_host_workspace_bytes": (sz, [vp, i32, i32, i32]),
+        "evk_retrieve_host": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, sz, vp]),
+        "evk_q_update_host_workspace_bytes": (sz, [vp, i64]),
+        "evk_q_update_host": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
+        "evk_last_status": (cint, [vp, vp]),
+        "evk_launch_count": (i64, [vp]),
+        "evk_strerror": (ctypes.c_char_p, [cint]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    return lib
+
+
+_lib = _load()
+
+
+def strerror(status: int) -> str:
+    return _lib.evk_strerror(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != EVK_OK:
+        raise EvkError(status, where)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _dev(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _host(t: torch.Tensor, dtype=None, name="tensor") -> int:
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _emb_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return EVK_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return EVK_DTYPE_BF16
+    raise ValueError(f"embeddings must be float32 or bfloat16, got {t.dtype}")
+
+
+class EvkMem:
+    """Handle of one memory bank: the opaque pointer plus the arena tensor that
+    backs it (kept alive here; the library does not own device memory)."""
+
+    def __init__(self, handle: int, arena: torch.Tensor, d: int, capacity: int, n_stages: int):
+        self.handle = handle
+        self.arena = arena
+        self.d, self.capacity, self.n_stages = d, capacity, n_stages
+        self._ws = {}
+
+    def workspace(self, kind: str, nbytes: int) -> torch.Tensor:
+        """A cached scratch tensor of at least nbytes on the arena's device."""
+        t = self._ws.get(kind)
+        if t is None or t.numel() < nbytes:
+            t = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.arena.device)
+            self._ws[kind] = t
+        return t
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h:
+            _lib.evk_mem_destroy(h)
+
+
+def evk_mem_bytes_required(d: int, capacity: int, n_stages: int = 2) -> int:
+    cfg = _Config(d, n_stages, capacity, 0.0, 0, None, 0)
+    n = _lib.evk_mem_bytes_required(ctypes.byref(cfg))
+    if n == 0:
+        raise EvkError(EVK_ERR_INVALID, "evk_mem_bytes_required")
+    return int(n)
+
+
+def evk_mem_create(d: int, capacity: int, n_stages: int = 2, q_default: float = 0.0,
+                   device="cuda", arena: Optional[torch.Tensor] = None) -> EvkMem:
+    nbytes = evk_mem_bytes_required(d, capacity, n_stages)
+    if arena is None:
+        arena = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    cfg = _Config(d, n_stages, capacity, q_default, 0, _dev(arena, torch.uint8, "arena"), arena.numel())
+    out = ctypes.c_void_p()
+    with torch.cuda.device(arena.device):
+        _check(_lib.evk_mem_create(ctypes.byref(cfg), ctypes.byref(out)), "evk_mem_create")
+    return EvkMem(out.value, arena, d, capacity, n_stages)
+
+
+def evk_mem_destroy(mem: EvkMem) -> None:
+    h, mem.handle = mem.handle, None
+    if h:
+        _check(_lib.evk_mem_destroy(h), "evk_mem_destroy")
+
+
+def evk_mem_size(mem: EvkMem) -> int:
+    return int(_lib.evk_mem_size(mem.handle))
+
+
+def evk_launch_count(mem: EvkMem) -> int:
+    return int(_lib.evk_launch_count(mem.handle))
+
+
+def evk_mem_set_scoring(mem: EvkMem, mode: int) -> None:
+    _check(_lib.evk_mem_set_scoring(mem.handle, mode), "evk_mem_set_scoring")
+
+
+def evk_mem_insert(mem: EvkMem, emb: torch.Tensor, stage: int = EVK_STAGE_ALL,
+                   q_init: Optional[torch.Tensor] = None, return_ids: bool = False, stream=None):
+    n = emb.shape[0]
+    if emb.dim() != 2 or emb.shape[1] != mem.d:
+        raise ValueError("emb must be [n][d]")
+    ids = torch.empty(n, dtype=torch.int32, device=emb.device) if return_ids else None
+    _check(_lib.evk_mem_insert(mem.handle, _dev(emb, None, "emb"), _emb_dtype(emb), n, stage,
+                               _dev(q_init, torch.float32, "q_init"), _dev(ids), _stream_ptr(stream)),
+           "evk_mem_insert")
+    return ids
+
+
+def evk_retrieve_workspace_bytes(mem: EvkMem, B: int, k1: int) -> int:
+    return int(_lib.evk_retrieve_workspace_bytes(mem.handle, B, k1))
+
+
+def evk_retrieve(mem: EvkMem, queries: torch.Tensor, stage: int, k1: int, k2: int, w: float,
+                 return_pool: bool = False, workspace: Optional[torch.Tensor] = None, stream=None,
+                 out=None):
+    """Returns (ids [B][k2] int32, scores [B][k2] fp32[, pool_ids, pool_sims])."""
+    if queries.dim() != 2 or queries.shape[1] != mem.d:
+        raise ValueError("queries must be [B][d]")
+    B = queries.shape[0]
+    dev = queries.device
+    if out is None:
+        ids = torch.empty((B, k2), dtype=torch.int32, device=dev)
+        scores = torch.empty((B, k2), dtype=torch.float32, device=dev)
+    else:
+        ids, scores = out
+    pool_ids = torch.empty((B, k1), dtype=torch.int32, device=dev) if return_pool else None
+    pool_sims = torch.empty((B, k1), dtype=torch.float32, device=dev) if return_pool else None
+    if workspace is None:
+        workspace = mem.workspace("retrieve", evk_retrieve_workspace_bytes(mem, B, k1))
+    _check(_lib.evk_retrieve(mem.handle, _dev(queries, None, "queries"), _emb_dtype(queries), B, stage,
+                             k1, k2, float(w), _dev(ids, torch.int32), _dev(scores, torch.float32),
+                             _dev(pool_ids), _dev(pool_sims),
+                             _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)),
+           "evk_retrieve")
+    if return_pool:
+        return ids, scores, pool_ids, pool_sims
+    return ids, scores
+
+
+def evk_q_update_workspace_bytes(mem: EvkMem, M: int) -> int:
+    return int(_lib.evk_q_update_workspace_bytes(mem.handle, M))
+
+
+def evk_q_update(mem: EvkMem, ids: torch.Tensor, stage: int, rewards: torch.Tensor, alpha: float,
+                 workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    M = ids.numel()
+    if rewards.numel() != M:
+        raise ValueError("ids and rewards must have the same length")
+    if workspace is None:
+        workspace = mem.workspace("q_update", evk_q_update_workspace_bytes(mem, M))
+    _check(_lib.evk_q_update(mem.handle, _dev(ids, torch.int32, "ids"), M, stage,
+                             _dev(rewards, torch.float32, "rewards"), float(alpha),
+                             _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)),
+           "evk_q_update")
+
+
+def evk_q_read(mem: EvkMem, stage: int, first: int = 0, n: Optional[int] = None, stream=None) -> torch.Tensor:
+    n = evk_mem_size(mem) - first if n is None else n
+    out = torch.empty(n, dtype=torch.float32, device=mem.arena.device)
+    _check(_lib.evk_q_read(mem.handle, stage, first, n, _dev(out), _stream_ptr(stream)), "evk_q_read")
+    return out
+
+
+def evk_q_write(mem: EvkMem, stage: int, values: torch.Tensor, first: int = 0, stream=None) -> None:
+    _check(_lib.evk_q_write(mem.handle, stage, first, values.numel(), _dev(values, torch.float32, "values"),
+                            _stream_ptr(stream)), "evk_q_write")
+
+
+def evk_bank_read(mem: EvkMem, first: int = 0, n: Optional[int] = None, stream=None) -> torch.Tensor:
+    n = evk_mem_size(mem) - first if n is None else n
+    out = torch.empty((n, mem.d), dtype=torch.bfloat16, device=mem.arena.device)
+    _check(_lib.evk_bank_read(mem.handle, first, n, _dev(out), _stream_ptr(stream)), "evk_bank_read")
+    return out
+
+
+def evk_retrieve_host(mem: EvkMem, queries_host: torch.Tensor, stage: int, k1: int, k2: int, w: float,
+                      ids_out_host: torch.Tensor, scores_out_host: torch.Tensor, stream=None) -> None:
+    """Host-buffer form: copies queries in and results out inside the call, then synchronises."""
+    B = queries_host.shape[0]
+    nbytes = int(_lib.evk_retrieve_host_workspace_bytes(mem.handle, B, k1, k2))
+    ws = mem.workspace("retrieve_host", nbytes)
+    _check(_lib.evk_retrieve_host(mem.handle, _host(queries_host, None, "queries_host"),
+                                  _emb_dtype(queries_host), B, stage, k1, k2, float(w),
+                                  _host(ids_out_host, torch.int32), _host(scores_out_host, torch.float32),
+                                  _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_retrieve_host")
+
+
+def evk_q_update_host(mem: EvkMem, ids_host: torch.Tensor, stage: int, rewards_host: torch.Tensor,
+                      alpha: float, stream=None) -> None:
+    M = ids_host.numel()
+    nbytes = int(_lib.evk_q_update_host_workspace_bytes(mem.handle, M))
+    ws = mem.workspace("q_update_host", nbytes)
+    _check(_lib.evk_q_update_host(mem.handle, _host(ids_host, torch.int32), M, stage,
+                                  _host(rewards_host, torch.float32), float(alpha),
+                                  _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_q_update_host")
+
+
+def evk_last_status(mem: EvkMem, stream=None) -> int:
+    return int(_lib.evk_last_status(mem.handle, _stream_ptr(stream)))

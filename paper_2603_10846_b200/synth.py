@@ -2,7 +2,7 @@
 
 This module only draws inputs (embeddings, queries, value tables, update
 batches).  It holds none of the retrieval or update arithmetic and is the one
-module that both the CUDA tests and the CPU oracle tests share.
+module shared by the CUDA path's tests and the CPU checker's tests.
 
 Large embedding matrices are drawn with a seeded ``torch.Generator`` on the
 device they are needed on (the bits differ between a CPU and a CUDA generator;

@@ -1,0 +1,356 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle, on the five
+synthetic bank shapes and on edge cases.  All tests here need a B200."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_10846_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def evk():
+    from paper_2603_10846_b200 import evk as _evk
+    return _evk
+
+
+def host_bits(t):
+    return synth.bf16_bits(t)
+
+
+def make_mem(evk, bank, q_tables, capacity=None, scoring=None):
+    """Create a bank, insert the rows (stage tables written afterwards), return the handle."""
+    n, d = bank.shape
+    mem = evk.evk_mem_create(d, capacity or max(n, 1), n_stages=q_tables.shape[0])
+    if scoring is not None:
+        evk.evk_mem_set_scoring(mem, scoring)
+    if n:
+        evk.evk_mem_insert(mem, bank)
+        for s in range(q_tables.shape[0]):
+            evk.evk_q_write(mem, s, torch.from_numpy(q_tables[s]).to(DEV))
+    return mem
+
+
+def run_retrieve(evk, mem, queries, stage, k1, k2, w):
+    out = evk.evk_retrieve(mem, queries, stage, k1, k2, w, return_pool=True)
+    torch.cuda.synchronize()
+    assert evk.evk_last_status(mem) == 0
+    return [x.cpu().numpy() for x in out]
+
+
+def sample_of(b, n, seed=0):
+    if b <= n:
+        return list(range(b))
+    return sorted(np.random.default_rng(seed).choice(b, n, replace=False).tolist())
+
+
+# ---------------------------------------------------------------------------
+# the five workloads
+# ---------------------------------------------------------------------------
+
+def test_tiny_fp32_bank_both_stages_then_updates(evk):
+    wl = synth.WORKLOADS["tiny"]
+    bank32 = synth.make_bank(wl, DEV)                       # fp32: the library rounds to bf16
+    queries32 = synth.make_queries(wl, wl.batches[0], DEV)
+    q_tab = synth.make_q_tables(wl)
+    mem = make_mem(evk, bank32, q_tab)
+    # the insert boundary: stored bits = the oracle's own nearest-even rounding
+    bank_bits = host_bits(evk.evk_bank_read(mem))
+    assert np.array_equal(bank_bits, oracle.bf16_round(bank32.cpu().numpy()))
+    q_bits = oracle.bf16_round(queries32.cpu().numpy())
+    for stage in (0, 1):
+        out = run_retrieve(evk, mem, queries32, stage, wl.k1, wl.k2, wl.w)
+        ep, ef = parity.check_retrieve(bank_bits, q_bits, q_tab[stage], wl.k1, wl.k2, wl.w, out)
+        assert ep == 1.0 and ef == 1.0
+    ids, r = synth.make_updates(wl)
+    evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 0, torch.from_numpy(r).to(DEV), wl.alpha)
+    q_after = evk.evk_q_read(mem, 0).cpu().numpy()
+    assert evk.evk_last_status(mem) == 0
+    parity.check_update(q_tab[0], ids, r, wl.alpha, q_after)
+    # the other stage's table keeps its bits, and its retrieval is unchanged
+    assert np.array_equal(evk.evk_q_read(mem, 1).cpu().numpy().view(np.uint32), q_tab[1].view(np.uint32))
+    out = run_retrieve(evk, mem, queries32, 0, wl.k1, wl.k2, wl.w)
+    parity.check_retrieve(bank_bits, q_bits, q_after, wl.k1, wl.k2, wl.w, out)
+
+
+def _workload_case(evk, name, b, n_oracle, stage=0, scoring=None, n=None):
+    wl = synth.WORKLOADS[name]
+    bank = synth.make_bank(wl, DEV, n=n)
+    queries = synth.make_queries(wl, b, DEV)
+    q_tab = synth.make_q_tables(wl, n=n)
+    mem = make_mem(evk, bank, q_tab, scoring=scoring)
+    out = run_retrieve(evk, mem, queries, stage, wl.k1, wl.k2, wl.w)
+    bank_bits, q_bits = host_bits(bank), host_bits(queries)
+    ep, ef = parity.check_retrieve(bank_bits, q_bits, q_tab[stage], wl.k1, wl.k2, wl.w, out,
+                                   sample=sample_of(b, n_oracle))
+    assert ep >= 0.9 and ef >= 0.9
+    return wl, mem, q_tab
+
+
+def test_mid_bank_retrieve_and_lognormal_updates(evk):
+    wl, mem, q_tab = _workload_case(evk, "mid", 256, 24, stage=1)
+    ids, r = synth.make_updates(wl)
+    evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 1, torch.from_numpy(r).to(DEV), wl.alpha)
+    parity.check_update(q_tab[1], ids, r, wl.alpha, evk.evk_q_read(mem, 1).cpu().numpy())
+
+
+def test_clustered_bank(evk):
+    _workload_case(evk, "clustered", 1024, 12)
+
+
+@pytest.mark.parametrize("b", [1, 8, 64])
+def test_large_bank_small_batches(evk, b):
+    _workload_case(evk, "large_hbm", b, 6)
+
+
+def test_large_bank_big_batch_with_zipf_updates(evk):
+    wl, mem, q_tab = _workload_case(evk, "large_compute", 4096, 4)
+    q = q_tab.copy()
+    for rnd in range(3):                       # streaming updates, stage alternating by round
+        stage = rnd % 2
+        ids, r = synth.make_updates(wl, round_idx=rnd)
+        evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), stage, torch.from_numpy(r).to(DEV), wl.alpha)
+        got = evk.evk_q_read(mem, stage).cpu().numpy()
+        parity.check_update(q[stage], ids, r, wl.alpha, got)
+        q[stage] = got
+    assert evk.evk_last_status(mem) == 0
+
+
+# ---------------------------------------------------------------------------
+# edge cases
+# ---------------------------------------------------------------------------
+
+def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None):
+    bank = synth.gaussian_unit(n, d, seed, DEV)
+    queries = synth.gaussian_unit(b, d, seed + 1, DEV)
+    q_tab = np.random.default_rng(seed).random((2, max(n, 1))).astype(np.float32)[:, :n]
+    mem = make_mem(evk, bank, np.ascontiguousarray(q_tab), capacity=capacity)
+    out = run_retrieve(evk, mem, queries, 0, k1, k2, w)
+    if n:
+        ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, k2, w, out)
+        assert ep >= 0.9 and ef >= 0.9
+    return mem, out
+
+
+@pytest.mark.parametrize("n,d,b,k1,k2", [
+    (1, 64, 3, 8, 2),            # single entry, pool mostly padding
+    (37, 8, 5, 64, 64),          # bank smaller than k1, narrowest rows, k2 = k1
+    (1000, 776, 7, 100, 10),     # width not a multiple of 256, ragged row count
+    (4097, 2048, 2, 1024, 16),   # widest rows, largest pool
+    (70001, 256, 9, 33, 5),      # several tiles per block plus a tail
+    (20000, 1024, 4, 1, 1),      # k1 = k2 = 1: plain argmax
+])
+def test_edge_shapes(evk, n, d, b, k1, k2):
+    _random_case(evk, n, d, b, k1, k2, 0.5, seed=n)
+
+
+def test_empty_bank_and_empty_batch(evk):
+    mem = evk.evk_mem_create(64, 128)
+    queries = synth.gaussian_unit(4, 64, 1, DEV)
+    ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, 16, 4, 0.5)
+    assert np.all(ids == -1) and np.all(np.isneginf(scores))
+    assert np.all(pool_ids == -1) and np.all(np.isneginf(pool_sims))
+    out = evk.evk_retrieve(mem, queries[:0], 0, 16, 4, 0.5)
+    assert out[0].shape == (0, 4)
+    evk.evk_q_update(mem, torch.empty(0, dtype=torch.int32, device=DEV), 0,
+                     torch.empty(0, dtype=torch.float32, device=DEV), 0.5)
+    assert evk.evk_last_status(mem) == 0
+
+
+def test_orthonormal_bank_is_exact(evk):
+    # sims are exact powers of two: no tolerance anywhere
+    d = 64
+    perm = np.random.default_rng(0).permutation(d)
+    bank = torch.eye(d, dtype=torch.float32)[perm].to(DEV)
+    q = (2.0 ** -torch.arange(d, dtype=torch.float32))[None, :].to(DEV)
+    mem = make_mem(evk, bank, np.zeros((2, d), np.float32))
+    ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, q, 0, 10, 10, 0.0)
+    inv = np.argsort(perm)
+    assert pool_ids[0].tolist() == [int(inv[i]) for i in range(10)]
+    assert pool_sims[0].tolist() == [2.0 ** -i for i in range(10)]
+    assert ids[0].tolist() == pool_ids[0].tolist()
+
+
+def test_ties_break_by_id_and_degenerate_scores(evk):
+    # duplicate rows tie exactly; a zero query makes every similarity equal
+    d, n = 128, 3000
+    bank = synth.gaussian_unit(n, d, 5, DEV)
+    bank[1234] = bank[17]
+    bank[2999] = bank[17]
+    q_tab = np.zeros((2, n), np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    queries = torch.cat([bank[17:18], torch.zeros((1, d), dtype=torch.bfloat16, device=DEV)])
+    ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, 40, 8, 0.0)
+    assert pool_ids[0, :3].tolist() == [17, 1234, 2999]
+    assert pool_ids[1].tolist() == list(range(40)) and np.all(pool_sims[1] == 0.0)
+    assert ids[1].tolist() == list(range(8))
+    parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], 40, 8, 0.0,
+                          (ids, scores, pool_ids, pool_sims))
+
+
+def test_bank_sorted_against_the_scan(evk):
+    # similarities increase with the row index, so every row beats the running threshold:
+    # the worst case for candidate-list upkeep.
+    d, n = 256, 50000
+    q = synth.gaussian_unit(1, d, 9, DEV)
+    bank = synth.gaussian_unit(n, d, 10, DEV)
+    sims = (bank.float() @ q.float().T).squeeze(1)
+    bank = bank[torch.argsort(sims)].contiguous()
+    q_tab = np.random.default_rng(1).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    out = run_retrieve(evk, mem, q, 1, 256, 16, 0.5)
+    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(q), q_tab[1], 256, 16, 0.5, out)
+    assert ep == 1.0
+
+
+def test_special_weights_and_stage_separation(evk):
+    n, d, b, k1, k2 = 5000, 128, 6, 32, 5
+    bank = synth.gaussian_unit(n, d, 21, DEV)
+    queries = synth.gaussian_unit(b, d, 22, DEV)
+    q_tab = np.random.default_rng(2).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    ids0, sc0, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, k1, k2, 0.0)
+    assert np.array_equal(ids0, pool_ids[:, :k2]) and np.array_equal(sc0, pool_sims[:, :k2])
+    for stage in (0, 1):
+        ids1, sc1, pool_ids1, _ = run_retrieve(evk, mem, queries, stage, k1, k2, 1.0)
+        assert np.array_equal(pool_ids1, pool_ids)      # the pool does not depend on the stage
+        for i in range(b):
+            order = np.argsort(-q_tab[stage][pool_ids[i]], kind="stable")[:k2]
+            assert ids1[i].tolist() == pool_ids[i][order].tolist()
+            assert np.array_equal(sc1[i], q_tab[stage][pool_ids[i][order]])
+    ids_all, _, _, _ = run_retrieve(evk, mem, queries, 0, k1, k1, 0.37)
+    assert np.array_equal(np.sort(ids_all, axis=1), np.sort(pool_ids, axis=1))
+    # an update of stage 0 cannot change a stage-1 retrieval
+    before = run_retrieve(evk, mem, queries, 1, k1, k2, 0.6)
+    upd = torch.arange(0, n, dtype=torch.int32, device=DEV)
+    evk.evk_q_update(mem, upd, 0, torch.ones(n, device=DEV), 0.5)
+    after = run_retrieve(evk, mem, queries, 1, k1, k2, 0.6)
+    for x, y in zip(before, after):
+        assert np.array_equal(x, y)
+
+
+def test_fp32_queries_equal_pre_rounded_bf16_queries(evk):
+    n, d = 3000, 512
+    bank = synth.gaussian_unit(n, d, 31, DEV)
+    q32 = synth.gaussian_unit(5, d, 32, DEV, dtype=torch.float32)
+    mem = make_mem(evk, bank, np.zeros((2, n), np.float32))
+    a = run_retrieve(evk, mem, q32, 0, 50, 7, 0.5)
+    b = run_retrieve(evk, mem, q32.to(torch.bfloat16), 0, 50, 7, 0.5)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
+def test_incremental_inserts_match_one_insert(evk):
+    n, d = 9000, 128
+    bank = synth.gaussian_unit(n, d, 41, DEV)
+    queries = synth.gaussian_unit(3, d, 42, DEV)
+    q0 = torch.rand(n, device=DEV)
+    whole = evk.evk_mem_create(d, n)
+    ids = evk.evk_mem_insert(whole, bank, evk.EVK_STAGE_DRAFT, q_init=q0, return_ids=True)
+    assert ids.cpu().tolist() == list(range(n))
+    parts = evk.evk_mem_create(d, n, q_default=0.25)
+    cuts = [0, 1, 64, 65, 4000, n]
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        evk.evk_mem_insert(parts, bank[a:b], evk.EVK_STAGE_DRAFT, q_init=q0[a:b])
+        assert evk.evk_mem_size(parts) == b
+        mid = run_retrieve(evk, parts, queries, 0, 16, 4, 0.5)          # cold start: sizes grow
+        assert np.all(mid[2][:, :min(16, b)] < b)
+    assert torch.equal(evk.evk_q_read(parts, 0), q0)
+    assert torch.all(evk.evk_q_read(parts, 1) == 0.25) and torch.all(evk.evk_q_read(whole, 1) == 0.0)
+    for x, y in zip(run_retrieve(evk, whole, queries, 0, 16, 4, 0.5),
+                    run_retrieve(evk, parts, queries, 0, 16, 4, 0.5)):
+        assert np.array_equal(x, y)
+    with pytest.raises(evk.EvkError) as e:
+        evk.evk_mem_insert(parts, bank[:1])
+    assert e.value.status == evk.EVK_ERR_CAPACITY
+
+
+def test_update_duplicates_split_and_order(evk):
+    n, m = 1000, 50000
+    rng = np.random.default_rng(51)
+    ids = np.where(rng.random(m) < 0.5, 7, rng.integers(0, n, m)).astype(np.int32)   # one very hot id
+    r = rng.standard_normal(m).astype(np.float32)
+    q0 = rng.standard_normal(n).astype(np.float32)
+    bank = synth.gaussian_unit(n, 64, 52, DEV)
+    results = []
+    for cuts in ([0, m], [0, 1, 2047, 2048, 2049, 30000, m]):
+        mem = make_mem(evk, bank, np.stack([q0, q0]))
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            evk.evk_q_update(mem, torch.from_numpy(ids[a:b]).to(DEV), 1, torch.from_numpy(r[a:b]).to(DEV), 0.3)
+        results.append(evk.evk_q_read(mem, 1).cpu().numpy())
+        assert evk.evk_last_status(mem) == 0
+    parity.check_update(q0, ids, r, 0.3, results[0])
+    assert np.array_equal(results[0].view(np.uint32), results[1].view(np.uint32))
+    # alpha = 1 is not special-cased: q + (r - q) in binary32
+    mem = make_mem(evk, bank, np.stack([q0, q0]))
+    evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 0, torch.from_numpy(r).to(DEV), 1.0)
+    parity.check_update(q0, ids, r, 1.0, evk.evk_q_read(mem, 0).cpu().numpy())
+
+
+def test_bad_updates_are_rejected_before_any_write(evk):
+    n = 500
+    bank = synth.gaussian_unit(n, 64, 61, DEV)
+    q0 = np.random.default_rng(3).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q0)
+    good = torch.arange(0, 100, dtype=torch.int32, device=DEV)
+    for bad_ids, bad_r, code in (
+            (torch.tensor([1, 2, n, 3], dtype=torch.int32), torch.zeros(4), evk.EVK_ERR_RANGE),
+            (torch.tensor([1, -1, 3], dtype=torch.int32), torch.zeros(3), evk.EVK_ERR_RANGE),
+            (torch.tensor([1, 2, 3], dtype=torch.int32), torch.tensor([0.0, float("nan"), 1.0]), evk.EVK_ERR_NONFINITE),
+            (torch.tensor([1, 2, 3], dtype=torch.int32), torch.tensor([0.0, float("inf"), 1.0]), evk.EVK_ERR_NONFINITE)):
+        evk.evk_q_update(mem, bad_ids.to(DEV), 0, bad_r.to(DEV), 0.5)
+        assert evk.evk_last_status(mem) == code
+        assert evk.evk_last_status(mem) == 0                       # read clears
+        assert np.array_equal(evk.evk_q_read(mem, 0).cpu().numpy().view(np.uint32), q0[0].view(np.uint32))
+    evk.evk_q_update(mem, good, 0, torch.ones(100, device=DEV), 0.5)       # the handle still works
+    assert evk.evk_last_status(mem) == 0
+    parity.check_update(q0[0], good.cpu().numpy(), np.ones(100, np.float32), 0.5,
+                        evk.evk_q_read(mem, 0).cpu().numpy())
+    # host-side argument checks return before anything is enqueued
+    queries = synth.gaussian_unit(2, 64, 62, DEV)
+    for kwargs in (dict(k1=8, k2=9, w=0.5), dict(k1=0, k2=1, w=0.5), dict(k1=2000, k2=1, w=0.5),
+                   dict(k1=8, k2=2, w=1.5), dict(k1=8, k2=2, w=-0.1)):
+        with pytest.raises(evk.EvkError) as e:
+            evk.evk_retrieve(mem, queries, 0, kwargs["k1"], kwargs["k2"], kwargs["w"])
+        assert e.value.status == evk.EVK_ERR_INVALID
+    for alpha in (0.0, -0.5, 1.5, float("nan")):
+        with pytest.raises(evk.EvkError):
+            evk.evk_q_update(mem, good, 0, torch.ones(100, device=DEV), alpha)
+    with pytest.raises(evk.EvkError):
+        evk.evk_retrieve(mem, queries, 2, 8, 2, 0.5)               # stage out of range
+
+
+def test_runs_are_bitwise_repeatable(evk):
+    n, d = 40000, 512
+    bank = synth.gaussian_unit(n, d, 71, DEV)
+    queries = synth.gaussian_unit(11, d, 72, DEV)
+    q_tab = np.random.default_rng(4).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    a = run_retrieve(evk, mem, queries, 0, 128, 8, 0.5)
+    for _ in range(3):
+        b = run_retrieve(evk, mem, queries, 0, 128, 8, 0.5)
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+
+
+def test_host_buffer_entry_points(evk):
+    n, d, b, k1, k2 = 20000, 256, 8, 64, 8
+    bank = synth.gaussian_unit(n, d, 81, DEV)
+    queries = synth.gaussian_unit(b, d, 82, DEV)
+    q_tab = np.random.default_rng(5).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    want = run_retrieve(evk, mem, queries, 0, k1, k2, 0.5)
+    q_host = queries.cpu().pin_memory()
+    ids_h = torch.empty((b, k2), dtype=torch.int32).pin_memory()
+    sc_h = torch.empty((b, k2), dtype=torch.float32).pin_memory()
+    evk.evk_retrieve_host(mem, q_host, 0, k1, k2, 0.5, ids_h, sc_h)
+    assert np.array_equal(ids_h.numpy(), want[0]) and np.array_equal(sc_h.numpy(), want[1])
+    ids = ids_h.reshape(-1).clone().pin_memory()
+    r = torch.ones(ids.numel()).pin_memory()
+    evk.evk_q_update_host(mem, ids, 0, r, 0.25)
+    parity.check_update(q_tab[0], ids.numpy(), r.numpy(), 0.25, evk.evk_q_read(mem, 0).cpu().numpy())
