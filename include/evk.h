@@ -165,6 +165,17 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
                       const float *rewards_host, float alpha,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* What evk_retrieve would run for a batch of B queries at the current size: the
+ * phase-1 kernel (EVK_SCORING_STREAM or EVK_SCORING_TENSOR) and how many times it
+ * is launched (each launch scans the whole bank once). */
+int evk_retrieve_plan(const evk_mem *mem, int32_t B, int32_t k1, int32_t *kind_out, int32_t *launches_out);
+
+/* Timing aid: the next evk_retrieve on this handle records `start_event` right
+ * before its phase-1 scoring launches and `stop_event` right after them, on that
+ * call's stream.  Both are cudaEvent_t owned by the caller, passed as void*.  The
+ * setting is used by one call and then cleared; NULLs clear it. */
+int evk_mem_profile_scoring(evk_mem *mem, void *start_event, void *stop_event);
+
 /* Synchronise `stream`, return the device status word (EVK_OK or the first
  * device-detected error since the last read) and clear it. */
 int evk_last_status(evk_mem *mem, void *stream);

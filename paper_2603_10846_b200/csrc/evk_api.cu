@@ -16,6 +16,7 @@ struct evk_mem {
     int32_t *status;      // device status word
     int scoring;
     int64_t launches;
+    cudaEvent_t prof_start, prof_stop;  // armed by evk_mem_profile_scoring for one retrieve
 };
 
 namespace {
@@ -91,6 +92,7 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     m->status = reinterpret_cast<int32_t *>(base + l.status);
     m->scoring = EVK_SCORING_AUTO;
     m->launches = 0;
+    m->prof_start = m->prof_stop = nullptr;
     cudaError_t err = cudaMemsetAsync(m->status, 0, 256, 0);
     if (err == cudaSuccess) err = cudaStreamSynchronize(0);
     if (err != cudaSuccess) {
@@ -173,12 +175,16 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     uint64_t *part_keys = reinterpret_cast<uint64_t *>(ws + l.part_keys);
 
     int nparts = 0;
+    cudaEvent_t ev_start = mem->prof_start, ev_stop = mem->prof_stop;
+    mem->prof_start = mem->prof_stop = nullptr;
+    if (err == cudaSuccess && ev_start) err = cudaEventRecord(ev_start, stream);
     if (err == cudaSuccess && mem->size > 0) {
         const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
         nparts = plan.nparts;
         err = launch_score_stream(mem->bank, mem->size, mem->cfg.d, q_bf16, B, k1, plan, part_keys,
                                   part_counts, stream, &launches);
     }
+    if (err == cudaSuccess && ev_stop) err = cudaEventRecord(ev_stop, stream);
     if (err == cudaSuccess)
         err = launch_merge_pool(part_keys, part_counts, nparts, k1, B, k1, pool_ids, pool_sims,
                                 pool_ids_out, pool_sims_out, stream, &launches);
@@ -187,6 +193,21 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
                             w, ids_out, scores_out, stream, &launches);
     mem->launches += launches;
     return cuda_status(err);
+}
+
+int evk_retrieve_plan(const evk_mem *mem, int32_t B, int32_t k1, int32_t *kind_out, int32_t *launches_out) {
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || !kind_out || !launches_out) return EVK_ERR_INVALID;
+    const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+    *kind_out = EVK_SCORING_STREAM;
+    *launches_out = (mem->size > 0 && B > 0) ? (B + plan.qb - 1) / plan.qb : 0;
+    return EVK_OK;
+}
+
+int evk_mem_profile_scoring(evk_mem *mem, void *start_event, void *stop_event) {
+    if (!mem) return EVK_ERR_INVALID;
+    mem->prof_start = static_cast<cudaEvent_t>(start_event);
+    mem->prof_stop = static_cast<cudaEvent_t>(stop_event);
+    return EVK_OK;
 }
 
 size_t evk_q_update_workspace_bytes(const evk_mem *mem, int64_t M) {

@@ -41,7 +41,8 @@ EXPORTS = (
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
-    "evk_q_update_host", "evk_last_status", "evk_launch_count", "evk_strerror",
+    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_last_status",
+    "evk_launch_count", "evk_strerror",
 )
 
 
@@ -84,6 +85,8 @@ def _load() -> ctypes.CDLL:
         "evk_retrieve_host": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, sz, vp]),
         "evk_q_update_host_workspace_bytes": (sz, [vp, i64]),
         "evk_q_update_host": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
+        "evk_retrieve_plan": (cint, [vp, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]),
+        "evk_mem_profile_scoring": (cint, [vp, vp, vp]),
         "evk_last_status": (cint, [vp, vp]),
         "evk_launch_count": (i64, [vp]),
         "evk_strerror": (ctypes.c_char_p, [cint]),
@@ -299,6 +302,22 @@ def evk_q_update_host(mem: EvkMem, ids_host: torch.Tensor, stage: int, rewards_h
     _check(_lib.evk_q_update_host(mem.handle, _host(ids_host, torch.int32), M, stage,
                                   _host(rewards_host, torch.float32), float(alpha),
                                   _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_q_update_host")
+
+
+def evk_retrieve_plan(mem: EvkMem, B: int, k1: int):
+    """(kernel kind, number of phase-1 launches) evk_retrieve would use at the current size."""
+    kind, launches = ctypes.c_int32(), ctypes.c_int32()
+    _check(_lib.evk_retrieve_plan(mem.handle, B, k1, ctypes.byref(kind), ctypes.byref(launches)),
+           "evk_retrieve_plan")
+    return kind.value, launches.value
+
+
+def evk_mem_profile_scoring(mem: EvkMem, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+    """Arm the next evk_retrieve to record these events around its phase-1 launches.
+    The events must already exist on the device (record them once before first use)."""
+    s = start.cuda_event if start is not None else None
+    e = stop.cuda_event if stop is not None else None
+    _check(_lib.evk_mem_profile_scoring(mem.handle, s, e), "evk_mem_profile_scoring")
 
 
 def evk_last_status(mem: EvkMem, stream=None) -> int:
