@@ -143,6 +143,35 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
                  const float *rewards, float alpha,
                  void *workspace, size_t workspace_bytes, void *stream);
 
+/* evk_q_update for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of the library.)
+ *
+ * Some hosts of this library cannot call cudaMalloc or grow a memory pool while
+ * they work: a serving loop whose device memory was carved up once at start-up and
+ * is fully spoken for, a plug-in running inside another framework's memory budget,
+ * a latency-critical section where an allocation (which may synchronise the device
+ * or fail) is not acceptable.  For them the scratch that the update's sort needs
+ * lives in a fixed array inside the library image instead of a caller workspace.
+ *
+ * Same arithmetic, order and error behaviour as evk_q_update; results are
+ * bit-identical.  Differences:
+ *   - M <= EVK_Q_UPDATE_STATIC_MAX; a larger batch returns EVK_ERR_UNSUPPORTED and
+ *     does nothing (split it: consecutive calls give the same bits as one call).
+ *   - About 1.06 MB of device memory is reserved on every GPU that loads the
+ *     library, for the life of the process, whether or not this call is used.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current, which it must be at every call); make that first call before
+ *     any stream capture begins.  The call itself allocates and frees nothing.
+ *   - Every call on a device shares the one array.  Calls are safe one after
+ *     another on one stream; two calls whose kernels can overlap on the GPU
+ *     (different streams without ordering) race on the scratch and corrupt each
+ *     other.  The array keeps the previous call's contents; the kernels clear or
+ *     overwrite everything they read.
+ * `ids` and `rewards` are device arrays as in evk_q_update. */
+enum { EVK_Q_UPDATE_STATIC_MAX = 65536 };
+int evk_q_update_static(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
+                        const float *rewards, float alpha, void *stream);
+
 /* Copy Q_stage[first .. first+n) to / from a device array. */
 int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream);
 int evk_q_write(evk_mem *mem, int stage, int64_t first, int64_t n, const float *values, void *stream);

@@ -231,6 +231,21 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
     return cuda_status(err);
 }
 
+int evk_q_update_static(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
+                        const float *rewards, float alpha, void *stream) {
+    if (!mem || M < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (!(alpha > 0.0f && alpha <= 1.0f)) return EVK_ERR_INVALID;
+    if (M == 0) return EVK_OK;
+    if (M > q_update_static_max()) return EVK_ERR_UNSUPPORTED;
+    if (!ids || !rewards) return EVK_ERR_INVALID;
+    int launches = 0;
+    cudaError_t err = launch_q_update_static(mem->q_tables + (size_t)stage * mem->cfg.capacity, mem->size, ids,
+                                             rewards, M, alpha, mem->status, static_cast<cudaStream_t>(stream),
+                                             &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
 int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream) {
     if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
     if (n == 0) return EVK_OK;

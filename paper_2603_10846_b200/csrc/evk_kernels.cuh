@@ -51,4 +51,9 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
                             int64_t m, float alpha, int32_t *status, void *workspace,
                             cudaStream_t stream, int *launches);
 
+// Eq. 4 update with scratch held in a static device array (no caller workspace).
+int64_t q_update_static_max();
+cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
+                                   int64_t m, float alpha, int32_t *status, cudaStream_t stream, int *launches);
+
 }  // namespace evk

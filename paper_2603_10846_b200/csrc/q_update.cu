@@ -12,6 +12,8 @@
 //
 // A checking pass runs first; if any id is out of range or any reward is not
 // finite, nothing is written and the status word records why.
+#include <mutex>
+
 #include "evk_common.cuh"
 #include "evk_kernels.cuh"
 
@@ -251,6 +253,53 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
     apply_kernel<<<(int)((m + kThreads - 1) / kThreads), kThreads, 0, stream>>>(k_in, v_in, m, alpha, q_stage, flags, status);
     ++*launches;
     return cudaGetLastError();
+}
+
+// ---- the same update for callers that cannot allocate device memory ------------
+//
+// Scratch for one batch of at most kStaticMaxUpdates updates, reserved in the
+// library image itself.  Every GPU that loads the library carries these bytes
+// until the process exits.  All calls on a device share the array.
+constexpr int64_t kStaticMaxUpdates = 65536;
+constexpr size_t kStaticScratchBytes = 256 + 256 * 32 * sizeof(int) + 4 * (size_t)kStaticMaxUpdates * 4;
+static __device__ __align__(256) unsigned char g_q_update_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_scratch_ptr[kMaxDevices];  // device address of g_q_update_scratch, per device ordinal
+std::mutex g_scratch_mu;
+
+// The array's name is only a host-side handle here; the address a kernel can use has to
+// be asked for, with the device that will run the kernel current.
+cudaError_t static_scratch(void **out) {
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    if (!g_scratch_ptr[dev]) {
+        void *p = nullptr;
+        err = cudaGetSymbolAddress(&p, g_q_update_scratch);
+        if (err != cudaSuccess) return err;
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
+int64_t q_update_static_max() { return kStaticMaxUpdates; }
+
+cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
+                                   int64_t m, float alpha, int32_t *status, cudaStream_t stream, int *launches) {
+    if (m <= 0) return cudaSuccess;
+    if (m > kStaticMaxUpdates || layout_for(m).total > kStaticScratchBytes) return cudaErrorInvalidValue;
+    void *scratch = nullptr;
+    cudaError_t err = static_scratch(&scratch);
+    if (err != cudaSuccess) return err;
+    // launch_q_update clears the flag word itself and overwrites every other part of the
+    // scratch it reads, so what the previous call left behind does not matter.
+    return launch_q_update(q_stage, size, ids, rewards, m, alpha, status, scratch, stream, launches);
 }
 
 }  // namespace evk

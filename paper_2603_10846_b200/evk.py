@@ -39,7 +39,7 @@ EVK_MAX_K1 = 1024
 EXPORTS = (
     "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
-    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_read", "evk_q_write", "evk_bank_read",
+    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_last_status",
     "evk_launch_count", "evk_strerror",
@@ -78,6 +78,7 @@ def _load() -> ctypes.CDLL:
         "evk_retrieve": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]),
         "evk_q_update_workspace_bytes": (sz, [vp, i64]),
         "evk_q_update": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
+        "evk_q_update_static": (cint, [vp, vp, i64, cint, vp, f32, vp]),
         "evk_q_read": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_q_write": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_bank_read": (cint, [vp, i64, i64, vp, vp]),
@@ -261,6 +262,23 @@ def evk_q_update(mem: EvkMem, ids: torch.Tensor, stage: int, rewards: torch.Tens
                              _dev(rewards, torch.float32, "rewards"), float(alpha),
                              _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)),
            "evk_q_update")
+
+
+EVK_Q_UPDATE_STATIC_MAX = 65536
+
+
+def evk_q_update_static(mem: EvkMem, ids: torch.Tensor, stage: int, rewards: torch.Tensor, alpha: float,
+                        stream=None) -> None:
+    """evk_q_update without a workspace: the sort's scratch is a fixed array inside the
+    library, so nothing is allocated here or in the library.  For callers whose device memory
+    is fully budgeted or who may not allocate while serving.  At most EVK_Q_UPDATE_STATIC_MAX
+    updates per call; calls on one device share the scratch and must not overlap on the GPU."""
+    M = ids.numel()
+    if rewards.numel() != M:
+        raise ValueError("ids and rewards must have the same length")
+    _check(_lib.evk_q_update_static(mem.handle, _dev(ids, torch.int32, "ids"), M, stage,
+                                    _dev(rewards, torch.float32, "rewards"), float(alpha), _stream_ptr(stream)),
+           "evk_q_update_static")
 
 
 def evk_q_read(mem: EvkMem, stage: int, first: int = 0, n: Optional[int] = None, stream=None) -> torch.Tensor:
