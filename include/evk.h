@@ -45,7 +45,9 @@ typedef enum evk_status {
     EVK_ERR_NONFINITE = -5,      /* device check: a reward that is NaN or infinite                    */
     EVK_ERR_DEVICE_TIMEOUT = -6, /* device: a bounded wait inside a kernel ran out                    */
     EVK_ERR_CUDA = -7,           /* a CUDA runtime or driver call failed                              */
-    EVK_ERR_UNSUPPORTED = -8     /* shape outside what the kernels support (see each call)            */
+    EVK_ERR_UNSUPPORTED = -8,    /* shape outside what the kernels support (see each call)            */
+    EVK_ERR_INCOMPLETE = -9      /* device check: a query found fewer candidates than min(k1, size),
+                                    which only non-finite similarities (NaN embeddings) can cause      */
 } evk_status;
 
 enum { EVK_DTYPE_F32 = 0, EVK_DTYPE_BF16 = 1 };

@@ -44,22 +44,43 @@ ArenaLayout arena_layout(const evk_config *c) {
 
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+// Which phase-1 kernel a batch goes to: EVK_SCORING_STREAM, EVK_SCORING_TENSOR, or 0 if the
+// forced kernel cannot take the shape.
+int pick_kind(const evk_mem *m, int32_t B, int32_t k1) {
+    const bool tensor_ok = mma_supported(m->cfg.d, k1);
+    const bool stream_ok = stream_supported(m->cfg.d);
+    if (m->scoring == EVK_SCORING_STREAM) return stream_ok ? EVK_SCORING_STREAM : 0;
+    if (m->scoring == EVK_SCORING_TENSOR) return tensor_ok ? EVK_SCORING_TENSOR : 0;
+    if (tensor_ok && B > 4) return EVK_SCORING_TENSOR;
+    return stream_ok ? EVK_SCORING_STREAM : (tensor_ok ? EVK_SCORING_TENSOR : 0);
+}
+
 struct RetrieveLayout {
-    size_t q_bf16, pool_ids, pool_sims, part_counts, part_keys, total;
+    size_t q_bf16, pool_ids, pool_sims, scratch, total;
+    size_t part_counts, part_keys;  // streaming kernel only, inside scratch
     int nparts_max;
 };
 
-RetrieveLayout retrieve_layout(const evk_mem *m, int32_t B, int32_t k1) {
+RetrieveLayout retrieve_layout(const evk_mem *m, int32_t B, int32_t k1, int kind) {
     RetrieveLayout l;
     const size_t b = (size_t)(B > 0 ? B : 0);
-    const StreamPlan plan = stream_plan(m->cfg.capacity, m->cfg.d, B, k1);
-    l.nparts_max = plan.nparts;
     l.q_bf16 = 0;
     l.pool_ids = l.q_bf16 + align256(b * m->cfg.d * sizeof(__nv_bfloat16));
     l.pool_sims = l.pool_ids + align256(b * k1 * sizeof(int32_t));
-    l.part_counts = l.pool_sims + align256(b * k1 * sizeof(float));
-    l.part_keys = l.part_counts + align256(b * l.nparts_max * sizeof(int));
-    l.total = l.part_keys + align256(b * l.nparts_max * (size_t)k1 * sizeof(uint64_t));
+    l.scratch = l.pool_sims + align256(b * k1 * sizeof(float));
+    l.part_counts = l.part_keys = 0;
+    l.nparts_max = 0;
+    size_t scratch_bytes = 256;
+    if (kind == EVK_SCORING_TENSOR) {
+        scratch_bytes = mma_workspace_bytes(B);
+    } else if (kind == EVK_SCORING_STREAM) {
+        const StreamPlan plan = stream_plan(m->cfg.capacity, m->cfg.d, B, k1);
+        l.nparts_max = plan.nparts;
+        l.part_counts = l.scratch;
+        l.part_keys = l.part_counts + align256(b * l.nparts_max * sizeof(int));
+        scratch_bytes = (l.part_keys - l.scratch) + align256(b * l.nparts_max * (size_t)k1 * sizeof(uint64_t));
+    }
+    l.total = l.scratch + scratch_bytes;
     return l;
 }
 
@@ -137,7 +158,7 @@ int evk_mem_insert(evk_mem *mem, const void *emb, int emb_dtype, int64_t n, int 
 
 size_t evk_retrieve_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1) {
     if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1) return 0;
-    return retrieve_layout(mem, B, k1).total + 256;
+    return retrieve_layout(mem, B, k1, pick_kind(mem, B, k1)).total + 256;
 }
 
 int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage,
@@ -152,10 +173,10 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     if (B == 0) return EVK_OK;
     if (!queries || !aligned(queries, 16) || !ids_out || !scores_out) return EVK_ERR_INVALID;
     if (!workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
-    const RetrieveLayout l = retrieve_layout(mem, B, k1);
+    const int kind = pick_kind(mem, B, k1);
+    if (kind == 0) return EVK_ERR_UNSUPPORTED;
+    const RetrieveLayout l = retrieve_layout(mem, B, k1, kind);
     if (workspace_bytes < l.total) return EVK_ERR_WORKSPACE;
-    if (mem->scoring == EVK_SCORING_TENSOR) return EVK_ERR_UNSUPPORTED;
-    if (!stream_supported(mem->cfg.d)) return EVK_ERR_UNSUPPORTED;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     char *ws = static_cast<char *>(workspace);
@@ -171,23 +192,43 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
 
     int32_t *pool_ids = reinterpret_cast<int32_t *>(ws + l.pool_ids);
     float *pool_sims = reinterpret_cast<float *>(ws + l.pool_sims);
-    int *part_counts = reinterpret_cast<int *>(ws + l.part_counts);
-    uint64_t *part_keys = reinterpret_cast<uint64_t *>(ws + l.part_keys);
-
-    int nparts = 0;
     cudaEvent_t ev_start = mem->prof_start, ev_stop = mem->prof_stop;
     mem->prof_start = mem->prof_stop = nullptr;
-    if (err == cudaSuccess && ev_start) err = cudaEventRecord(ev_start, stream);
+
+    // phase 1: per-(query, part) candidate lists, then one merge per query
+    const uint64_t *part_keys = nullptr;
+    const int *part_counts = nullptr;
+    int nparts = 0, part_stride = k1, qt_size = 1;
     if (err == cudaSuccess && mem->size > 0) {
-        const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
-        nparts = plan.nparts;
-        err = launch_score_stream(mem->bank, mem->size, mem->cfg.d, q_bf16, B, k1, plan, part_keys,
-                                  part_counts, stream, &launches);
+        if (kind == EVK_SCORING_TENSOR) {
+            const MmaPlan plan = mma_plan(mem->size, B, k1);
+            uint64_t *cand = nullptr;
+            int *cand_cnt = nullptr;
+            err = launch_score_mma(mem->bank, mem->size, mem->cfg.capacity, mem->cfg.d, q_bf16, B, k1, plan,
+                                   ws + l.scratch, mem->status, &cand, &cand_cnt, ev_start, ev_stop, stream, &launches);
+            part_keys = cand;
+            part_counts = cand_cnt;
+            nparts = plan.splits;
+            part_stride = kMmaCandCap;
+            qt_size = 128;
+        } else {
+            const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+            uint64_t *keys = reinterpret_cast<uint64_t *>(ws + l.part_keys);
+            int *counts = reinterpret_cast<int *>(ws + l.part_counts);
+            if (ev_start) err = cudaEventRecord(ev_start, stream);
+            if (err == cudaSuccess)
+                err = launch_score_stream(mem->bank, mem->size, mem->cfg.d, q_bf16, B, k1, plan, keys, counts,
+                                          stream, &launches);
+            if (err == cudaSuccess && ev_stop) err = cudaEventRecord(ev_stop, stream);
+            part_keys = keys;
+            part_counts = counts;
+            nparts = plan.nparts;
+        }
     }
-    if (err == cudaSuccess && ev_stop) err = cudaEventRecord(ev_stop, stream);
+    const int expect = (int)(mem->size < k1 ? mem->size : k1);
     if (err == cudaSuccess)
-        err = launch_merge_pool(part_keys, part_counts, nparts, k1, B, k1, pool_ids, pool_sims,
-                                pool_ids_out, pool_sims_out, stream, &launches);
+        err = launch_merge_pool(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect, mem->status,
+                                pool_ids, pool_sims, pool_ids_out, pool_sims_out, stream, &launches);
     if (err == cudaSuccess)
         err = launch_rerank(pool_ids, pool_sims, B, k1, k2, mem->q_tables + (size_t)stage * mem->cfg.capacity,
                             w, ids_out, scores_out, stream, &launches);
@@ -197,9 +238,17 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
 
 int evk_retrieve_plan(const evk_mem *mem, int32_t B, int32_t k1, int32_t *kind_out, int32_t *launches_out) {
     if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || !kind_out || !launches_out) return EVK_ERR_INVALID;
-    const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
-    *kind_out = EVK_SCORING_STREAM;
-    *launches_out = (mem->size > 0 && B > 0) ? (B + plan.qb - 1) / plan.qb : 0;
+    const int kind = pick_kind(mem, B, k1);
+    if (kind == 0) return EVK_ERR_UNSUPPORTED;
+    *kind_out = kind;
+    if (mem->size <= 0 || B <= 0) {
+        *launches_out = 0;
+    } else if (kind == EVK_SCORING_TENSOR) {
+        *launches_out = 1;
+    } else {
+        const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+        *launches_out = (B + plan.qb - 1) / plan.qb;
+    }
     return EVK_OK;
 }
 
@@ -359,6 +408,7 @@ const char *evk_strerror(int status) {
         case EVK_ERR_DEVICE_TIMEOUT: return "bounded wait in a kernel ran out";
         case EVK_ERR_CUDA: return "CUDA call failed";
         case EVK_ERR_UNSUPPORTED: return "unsupported shape";
+        case EVK_ERR_INCOMPLETE: return "fewer candidates than min(k1, size): non-finite similarities";
         default: return "unknown status";
     }
 }

@@ -33,10 +33,35 @@ cudaError_t launch_score_stream(const __nv_bfloat16 *bank, int64_t size, int d,
                                 const __nv_bfloat16 *queries, int B, int k1, const StreamPlan &plan,
                                 uint64_t *part_keys, int *part_counts, cudaStream_t stream, int *launches);
 
+// ---- phase 1, tensor-core kernel ---------------------------------------------
+// Candidate lists: job = query_tile * splits + split; list = job * 128 + (query % 128);
+// cand_cnt[list] keys at cand[list * kMmaCandCap ...].
+constexpr int kMmaCandCap = 1024;  // keys per candidate list
+constexpr int kMmaSample = 4096;   // bank rows sampled for the starting thresholds
+struct MmaPlan {
+    int n_qt;               // query tiles of 128
+    int n_tiles;            // bank tiles of 256 rows
+    int splits;             // bank splits per query tile (= candidate lists per query)
+    int grid;               // thread blocks
+    int n_sample;           // 0: no sampling pass
+    int64_t sample_stride;  // rows between sampled entries
+};
+bool mma_supported(int d, int k1);
+MmaPlan mma_plan(int64_t size, int B, int k1);
+size_t mma_workspace_bytes(int B);
+// ev_start / ev_stop (may be null) are recorded around the full-bank launch only.
+cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t capacity, int d,
+                             const __nv_bfloat16 *queries, int B, int k1, const MmaPlan &plan, void *workspace,
+                             int32_t *status, uint64_t **cand_out, int **cand_cnt_out,
+                             cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream, int *launches);
+
 // ---- phase 1, pool merge ----------------------------------------------------
+// List of (query q, part p): (q / qt_size) * (nparts * qt_size) + p * qt_size + q % qt_size.
+// expect: entries every query must at least have (min(k1, size)); fewer sets EVK_ERR_INCOMPLETE.
 constexpr int kMergeMaxParts = 2048;
 cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
-                              int part_stride, int B, int k1, int32_t *pool_ids, float *pool_sims,
+                              int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                              int32_t *pool_ids, float *pool_sims,
                               int32_t *pool_ids_user, float *pool_sims_user,
                               cudaStream_t stream, int *launches);
 

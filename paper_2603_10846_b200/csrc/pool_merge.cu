@@ -21,7 +21,8 @@ constexpr int kBatch = 2048;                    // candidates examined between c
 
 __global__ void __launch_bounds__(kThreads)
 merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
-                  int part_stride, int k1, int32_t *__restrict__ pool_ids, float *__restrict__ pool_sims,
+                  int part_stride, int qt_size, int k1, int expect, int32_t *__restrict__ status,
+                  int32_t *__restrict__ pool_ids, float *__restrict__ pool_sims,
                   int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user) {
     __shared__ __align__(16) uint64_t keys[kCap];
     __shared__ int offs[kMergeMaxParts + 1];
@@ -32,7 +33,8 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
 
     const int tid = threadIdx.x;
     const int q = blockIdx.x;
-    const int *cnt = part_counts + (size_t)q * nparts;
+    // list of part p: list0 + p * qt_size
+    const size_t list0 = (size_t)(q / qt_size) * ((size_t)nparts * qt_size) + (size_t)(q % qt_size);
 
     // exclusive scan of the part counts (single thread per 8 parts, then serial over chunks:
     // nparts is at most a few thousand)
@@ -40,7 +42,7 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
         count = 0;
         tau = 0;
     }
-    for (int p = tid; p < nparts; p += kThreads) offs[p + 1] = cnt[p];
+    for (int p = tid; p < nparts; p += kThreads) offs[p + 1] = part_counts[list0 + (size_t)p * qt_size];
     if (tid == 0) offs[0] = 0;
     __syncthreads();
     if (tid < 32) {
@@ -73,7 +75,7 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
                     const int mid = (lo + hi) >> 1;
                     if (offs[mid] <= idx) lo = mid; else hi = mid;
                 }
-                const uint64_t key = part_keys[((size_t)q * nparts + lo) * part_stride + (idx - offs[lo])];
+                const uint64_t key = part_keys[(list0 + (size_t)lo * qt_size) * part_stride + (idx - offs[lo])];
                 if (key > t) keys[atomicAdd(&count, 1)] = key;
             }
         }
@@ -90,6 +92,7 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
     }
 
     int n = count;
+    if (n < expect && tid == 0) atomicCAS(status, 0, (int)EVK_ERR_INCOMPLETE);
     if (n > k1) {
         block_select_topk<kThreads, kSelPerThread>(keys, n, k1, hist, scal);
         n = k1;
@@ -115,13 +118,14 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
 }  // namespace
 
 cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
-                              int part_stride, int B, int k1, int32_t *pool_ids, float *pool_sims,
+                              int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                              int32_t *pool_ids, float *pool_sims,
                               int32_t *pool_ids_user, float *pool_sims_user,
                               cudaStream_t stream, int *launches) {
     if (B <= 0) return cudaSuccess;
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
-    merge_pool_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, k1,
-                                                  pool_ids, pool_sims, pool_ids_user, pool_sims_user);
+    merge_pool_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, qt_size, k1, expect,
+                                                  status, pool_ids, pool_sims, pool_ids_user, pool_sims_user);
     ++*launches;
     return cudaGetLastError();
 }

@@ -1,0 +1,586 @@
+// Phase 1 on the tensor cores: similarity of a tile of 128 queries against the
+// whole bank as a bf16 GEMM with fp32 accumulation (tcgen05.mma, accumulators in
+// tensor memory), with the top-k1 selection fused into the epilogue so that the
+// B x N similarity matrix of Section 3.2's dense retrieval is never written out.
+//
+// Layout of one thread block (192 threads, one block per SM, persistent):
+//   warp 0     TMA producer: streams 64-column slices of the query tile (A, 128 rows)
+//              and of a bank tile (B, 256 rows) into a 4-stage shared-memory ring,
+//              128-byte swizzled, K-major.
+//   warp 1     MMA issuer: one thread issues tcgen05.mma 128x256x16 per 16 columns of
+//              a slice, accumulating D[query][bank row] in one of two 256-column
+//              tensor-memory buffers; tcgen05.commit hands smem stages back to the
+//              producer and finished accumulators to the epilogue.
+//   warps 2-5  epilogue: thread m owns query m of the tile (= TMEM lane m).  It reads
+//              its 256 similarities of a bank tile 32 at a time, compares them with
+//              the query's running threshold held in a register, and appends the few
+//              survivors to the query's private candidate list in global memory.
+//              When a list fills, the warp cuts it back to its best k1 with an exact
+//              radix select over registers and the threshold rises.
+//
+// A bank tile is 256 consecutive entries; the queries sit on the accumulator's
+// lanes so that the per-query threshold test costs one register compare and no
+// cross-thread traffic.  The work of a launch is a grid of jobs (query tile,
+// bank split); the bank tiles of a split are interleaved (t = split, split+S, ...)
+// so that blocks working on different query tiles touch the same bank tile at about
+// the same time and share it through L2.
+//
+// The same kernel has a "dense" mode that writes every similarity of a small,
+// strided sample of the bank; its k1-th largest value per query is a safe starting
+// threshold for the full scan (at least k1 entries of the bank reach it).
+//
+// Every wait on an mbarrier is bounded; a wait that runs out raises the block's
+// abort flag, every role leaves its loop, tensor memory is released and the status
+// word reports EVK_ERR_DEVICE_TIMEOUT.
+#include <cuda.h>
+
+#include "evk_common.cuh"
+#include "evk_kernels.cuh"
+
+namespace evk {
+
+namespace {
+
+constexpr int kBlockM = 128;
+constexpr int kBlockN = 256;
+constexpr int kBlockK = 64;
+constexpr int kUmmaK = 16;
+constexpr int kStages = 4;
+constexpr int kThreads = 192;
+constexpr uint32_t kABytes = kBlockM * kBlockK * 2;  // 16 KB
+constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;  // 32 KB
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kTmemCols = 512;                  // two accumulators of 256 fp32 columns
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
+
+// tcgen05 instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=256, M=128.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
+                                ((uint32_t)(kBlockM >> 4) << 24);
+
+struct MmaParams {
+    int64_t size;       // valid bank rows (filter mode) or sample rows (dense mode)
+    int B, d, k1;
+    int n_qt, splits, n_tiles;
+    int mode;           // 0 = filter, 1 = dense
+    const float *tau0;  // [B] starting thresholds, or nullptr
+    uint64_t *cand;     // [n_qt*splits][128][kMmaCandCap]
+    int *cand_cnt;      // [n_qt*splits][128]
+    float *dense;       // [B][dense_ld]
+    int dense_ld;
+    int32_t *status;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false means the block is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kTimeoutCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- warp-wide exact selection over one candidate list ------------------------
+// The whole warp cuts the list `buf` (n <= kMmaCandCap distinct non-zero keys) back to
+// its k largest and returns the k-th largest key.  Keys live in registers (32 per
+// lane); the k-th largest is found 4 bits at a time from the top.
+__device__ __noinline__ uint64_t warp_select_topk(uint64_t *buf, int n, int k) {
+    const int lane = threadIdx.x & 31;
+    constexpr int kPerLane = kMmaCandCap / 32;
+    uint64_t r[kPerLane];
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) {
+        const int i = j * 32 + lane;
+        r[j] = (i < n) ? buf[i] : 0;
+    }
+    uint64_t prefix = 0, mask = 0;
+    int kk = k;
+#pragma unroll 1
+    for (int shift = 60; shift >= 0; shift -= 4) {
+        // per-lane counts of the 16 digit values, 8 bits each (a lane holds at most 32 keys)
+        uint64_t c_lo = 0, c_hi = 0;
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+            if ((r[j] & mask) == prefix && r[j] != 0) {
+                const int dgt = (int)((r[j] >> shift) & 15);
+                if (dgt < 8) c_lo += (uint64_t)1 << (8 * dgt);
+                else c_hi += (uint64_t)1 << (8 * (dgt - 8));
+            }
+        }
+        int acc = 0, digit = 0;
+        bool found = false;
+#pragma unroll
+        for (int b = 15; b >= 0; --b) {
+            const uint32_t mine = (uint32_t)(((b < 8) ? (c_lo >> (8 * b)) : (c_hi >> (8 * (b - 8)))) & 0xff);
+            const int cnt = (int)__reduce_add_sync(0xffffffffu, mine);
+            if (!found) {
+                if (kk <= acc + cnt) {
+                    digit = b;
+                    found = true;
+                } else {
+                    acc += cnt;
+                }
+            }
+        }
+        kk -= acc;
+        prefix |= (uint64_t)digit << shift;
+        mask |= (uint64_t)15 << shift;
+    }
+    // prefix is the k-th largest key; exactly k keys are >= prefix.  Compact in place.
+    int keep = 0;
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) keep += (r[j] >= prefix && r[j] != 0);
+    int start = keep;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, start, off);
+        if (lane >= off) start += v;
+    }
+    start -= keep;
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j)
+        if (r[j] >= prefix && r[j] != 0) buf[start++] = r[j];
+    __syncwarp();
+    return prefix;
+}
+
+// ---- the kernel ---------------------------------------------------------------
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
+                 const MmaParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the swizzled tiles
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    unsigned char *tiles_ptr = smem_raw + (tiles - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tiles_ptr + (size_t)kStages * kStageBytes);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
+    const uint32_t tfull0 = empty0 + 8 * kStages, tempty0 = tfull0 + 16;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull0 + 8 * b, 1);
+            mbar_init(tempty0 + 8 * b, 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_jobs = p.n_qt * p.splits;
+    const int k_chunks = p.d / kBlockK;
+
+    if (warp == 0) {
+        // ===== TMA producer =====
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+                const int qt = job / p.splits, split = job % p.splits;
+                for (int t = split; t < p.n_tiles && ok; t += p.splits) {
+                    for (int kc = 0; kc < k_chunks; ++kc) {
+                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t a_dst = tiles + stage * kStageBytes;
+                        const uint32_t b_dst = a_dst + kABytes;
+                        mbar_arrive_expect_tx(full0 + 8 * stage, kStageBytes);
+                        tma_load_2d(a_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
+                        tma_load_2d(b_dst, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
+                        if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===== MMA issuer =====
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+                const int split = job % p.splits;
+                for (int t = split; t < p.n_tiles && ok; t += p.splits) {
+                    if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * kBlockN;
+                    for (int kc = 0; kc < k_chunks; ++kc) {
+                        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles + stage * kStageBytes;
+                        const uint64_t a_desc = smem_desc(a_addr);
+                        const uint64_t b_desc = smem_desc(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                            // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
+                            umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                      (kc > 0 || k > 0) ? 1u : 0u);
+                        }
+                        umma_commit(empty0 + 8 * stage);
+                        if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    }
+                    if (!ok) break;
+                    umma_commit(tfull0 + 8 * acc);
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                }
+            }
+        }
+    } else {
+        // ===== epilogue: thread = one query of the tile = one TMEM lane =====
+        const int quarter = warp & 3;              // warps 2,3,4,5 -> lane quarters 2,3,0,1
+        const int m = quarter * 32 + lane;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+            const int qt = job / p.splits, split = job % p.splits;
+            const int q = qt * kBlockM + m;
+            const bool q_valid = q < p.B;
+            float tau_sim = INFINITY;
+            uint64_t tau_key = ~(uint64_t)0;
+            if (q_valid) {
+                if (p.tau0) {
+                    // every entry whose similarity reaches the sampled threshold passes
+                    tau_sim = p.tau0[q];
+                    tau_key = (uint64_t)ordered_bits(tau_sim + 0.0f) << 32;
+                } else {
+                    tau_sim = -INFINITY;
+                    tau_key = 0;
+                }
+            }
+            int cnt = 0;
+            uint64_t *my_buf = p.cand + ((size_t)job * kBlockM + m) * kMmaCandCap;
+            for (int t = split; t < p.n_tiles && ok; t += p.splits) {
+                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
+                const int64_t row0 = (int64_t)t * kBlockN;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kBlockN; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(t_addr + c0, v);
+                    if (p.mode == 1) {
+                        if (q_valid) {
+                            float4 *dst = reinterpret_cast<float4 *>(p.dense + (size_t)q * p.dense_ld + row0 + c0);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        }
+                        continue;
+                    }
+                    float mx = __uint_as_float(v[0]);
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
+                    if (mx >= tau_sim) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float s = __uint_as_float(v[j]);
+                            const int64_t row = row0 + c0 + j;
+                            if (s >= tau_sim && row < p.size) {
+                                const uint64_t key = make_key(s, (int32_t)row);
+                                if (key > tau_key) my_buf[cnt++] = key;
+                            }
+                        }
+                    }
+                    // lists that could overflow on the next 32 columns are cut back to their best k1
+                    uint32_t need = __ballot_sync(0xffffffffu, cnt > kMmaCandCap - 32);
+                    while (need) {
+                        const int owner = __ffs(need) - 1;
+                        need &= need - 1;
+                        const int n = __shfl_sync(0xffffffffu, cnt, owner);
+                        uint64_t *buf = reinterpret_cast<uint64_t *>(
+                            __shfl_sync(0xffffffffu, (unsigned long long)my_buf, owner));
+                        __syncwarp();
+                        const uint64_t kth = warp_select_topk(buf, n, p.k1);
+                        if (lane == owner) {
+                            cnt = p.k1;
+                            tau_key = kth;
+                            tau_sim = key_sim(kth);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+            if (p.mode == 0 && ok) p.cand_cnt[(size_t)job * kBlockM + m] = cnt;
+        }
+    }
+
+    // ===== teardown =====
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies still in flight time to land before shared memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)EVK_ERR_DEVICE_TIMEOUT);
+        __syncthreads();
+    }
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// k1-th largest of each query's sample similarities -> starting threshold.
+constexpr int kSelThreads = 512;
+constexpr int kSelPerThread = kMmaSample / kSelThreads;
+
+__global__ void __launch_bounds__(kSelThreads)
+sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0) {
+    __shared__ uint64_t keys[kMmaSample];
+    __shared__ int hist[256];
+    __shared__ uint64_t scal[4];
+    const int q = blockIdx.x;
+    for (int i = threadIdx.x; i < n_sample; i += kSelThreads) keys[i] = make_key(dense[(size_t)q * ld + i], i);
+    __syncthreads();
+    const uint64_t kth = block_select_topk<kSelThreads, kSelPerThread>(keys, n_sample, k1, hist, scal);
+    if (threadIdx.x == 0) tau0[q] = key_sim(kth);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// A [rows][d] bf16 matrix whose consecutive rows are row_stride_elems apart, boxed 64 x box_rows.
+bool make_map(CUtensorMap *map, const void *base, int d, int64_t rows, int64_t row_stride_elems, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)row_stride_elems * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
+                          cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    score_mma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mq, mb, p);
+    return cudaGetLastError();
+}
+
+struct MmaLayout {
+    size_t cand, cand_cnt, dense, tau0, total;
+};
+
+MmaLayout mma_layout(int B) {
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t n_qt = (size_t)((B + kBlockM - 1) / kBlockM);
+    // jobs = n_qt * floor(148 / n_qt) <= 148 while n_qt <= 148, else one split per query tile
+    const size_t lists = (n_qt > (size_t)kNumSM ? n_qt : (size_t)kNumSM) * kBlockM;
+    MmaLayout l;
+    l.cand = 0;
+    l.cand_cnt = l.cand + align(lists * kMmaCandCap * sizeof(uint64_t));
+    l.dense = l.cand_cnt + align(lists * sizeof(int));
+    l.tau0 = l.dense + align(n_qt * kBlockM * kMmaSample * sizeof(float));
+    l.total = l.tau0 + align(n_qt * kBlockM * sizeof(float));
+    return l;
+}
+
+int splits_for(int n_qt, int n_tiles) {
+    int splits = kNumSM / (n_qt > 0 ? n_qt : 1);
+    if (splits < 1) splits = 1;
+    if (splits > n_tiles) splits = n_tiles > 0 ? n_tiles : 1;
+    return splits;
+}
+
+}  // namespace
+
+bool mma_supported(int d, int k1) {
+    return d % kBlockK == 0 && d >= kBlockK && k1 <= kMmaCandCap / 2 && encode_fn() != nullptr;
+}
+
+MmaPlan mma_plan(int64_t size, int B, int k1) {
+    MmaPlan pl;
+    pl.n_qt = (B + kBlockM - 1) / kBlockM;
+    pl.n_tiles = (int)((size + kBlockN - 1) / kBlockN);
+    pl.splits = splits_for(pl.n_qt, pl.n_tiles);
+    const int jobs = pl.n_qt * pl.splits;
+    pl.grid = jobs < kNumSM ? jobs : kNumSM;
+    if (pl.grid < 1) pl.grid = 1;
+    // a strided sample of the bank gives each query a starting threshold
+    pl.n_sample = (size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
+    pl.sample_stride = pl.n_sample ? size / pl.n_sample : 0;
+    return pl;
+}
+
+size_t mma_workspace_bytes(int B) { return mma_layout(B).total; }
+
+cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t capacity, int d,
+                             const __nv_bfloat16 *queries, int B, int k1, const MmaPlan &pl, void *workspace,
+                             int32_t *status, uint64_t **cand_out, int **cand_cnt_out,
+                             cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream, int *launches) {
+    const MmaLayout l = mma_layout(B);
+    char *ws = static_cast<char *>(workspace);
+    uint64_t *cand = reinterpret_cast<uint64_t *>(ws + l.cand);
+    int *cand_cnt = reinterpret_cast<int *>(ws + l.cand_cnt);
+    float *dense = reinterpret_cast<float *>(ws + l.dense);
+    float *tau0 = reinterpret_cast<float *>(ws + l.tau0);
+    *cand_out = cand;
+    *cand_cnt_out = cand_cnt;
+
+    CUtensorMap map_q, map_bank;
+    if (!make_map(&map_q, queries, d, B, d, kBlockM)) return cudaErrorInvalidValue;
+
+    MmaParams p;
+    p.B = B;
+    p.d = d;
+    p.k1 = k1;
+    p.n_qt = pl.n_qt;
+    p.cand = cand;
+    p.cand_cnt = cand_cnt;
+    p.dense = dense;
+    p.dense_ld = kMmaSample;
+    p.status = status;
+    p.tau0 = nullptr;
+
+    if (pl.n_sample) {
+        // dense pass over every sample_stride-th row
+        CUtensorMap map_sample;
+        if (!make_map(&map_sample, bank, d, pl.n_sample, pl.sample_stride * d, kBlockN)) return cudaErrorInvalidValue;
+        p.size = pl.n_sample;
+        p.mode = 1;
+        p.n_tiles = pl.n_sample / kBlockN;
+        p.splits = splits_for(p.n_qt, p.n_tiles);
+        const int jobs = p.n_qt * p.splits;
+        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, stream);
+        if (err != cudaSuccess) return err;
+        ++*launches;
+        sample_threshold_kernel<<<B, kSelThreads, 0, stream>>>(dense, kMmaSample, pl.n_sample, k1, tau0);
+        err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        ++*launches;
+        p.tau0 = tau0;
+    }
+
+    if (!make_map(&map_bank, bank, d, capacity, d, kBlockN)) return cudaErrorInvalidValue;
+    p.size = size;
+    p.mode = 0;
+    p.n_tiles = pl.n_tiles;
+    p.splits = pl.splits;
+    cudaError_t err = cudaSuccess;
+    if (ev_start) err = cudaEventRecord(ev_start, stream);
+    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, stream);
+    if (err != cudaSuccess) return err;
+    ++*launches;
+    if (ev_stop) err = cudaEventRecord(ev_stop, stream);
+    return err;
+}
+
+}  // namespace evk

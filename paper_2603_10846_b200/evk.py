@@ -29,6 +29,7 @@ EVK_ERR_NONFINITE = -5
 EVK_ERR_DEVICE_TIMEOUT = -6
 EVK_ERR_CUDA = -7
 EVK_ERR_UNSUPPORTED = -8
+EVK_ERR_INCOMPLETE = -9
 
 EVK_DTYPE_F32, EVK_DTYPE_BF16 = 0, 1
 EVK_STAGE_DRAFT, EVK_STAGE_REFINE, EVK_STAGE_ALL = 0, 1, -1

@@ -49,7 +49,8 @@ def test_sizes_and_messages_without_a_device(lib_path):
             evk.evk_mem_bytes_required(*bad)
     assert evk.strerror(0) == "ok"
     codes = [evk.EVK_ERR_INVALID, evk.EVK_ERR_CAPACITY, evk.EVK_ERR_WORKSPACE, evk.EVK_ERR_RANGE,
-             evk.EVK_ERR_NONFINITE, evk.EVK_ERR_DEVICE_TIMEOUT, evk.EVK_ERR_CUDA, evk.EVK_ERR_UNSUPPORTED]
+             evk.EVK_ERR_NONFINITE, evk.EVK_ERR_DEVICE_TIMEOUT, evk.EVK_ERR_CUDA, evk.EVK_ERR_UNSUPPORTED,
+             evk.EVK_ERR_INCOMPLETE]
     assert len({evk.strerror(c) for c in codes}) == len(codes)
     # null handles are refused, not dereferenced
     assert evk._lib.evk_mem_size(None) == 0

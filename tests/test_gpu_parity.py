@@ -19,6 +19,16 @@ def evk():
     return _evk
 
 
+@pytest.fixture(params=["stream", "tensor"])
+def scoring(request, evk):
+    """Both phase-1 kernels are forced in turn."""
+    return {"stream": evk.EVK_SCORING_STREAM, "tensor": evk.EVK_SCORING_TENSOR}[request.param]
+
+
+def tensor_unsupported(evk, scoring, d, k1):
+    return scoring == evk.EVK_SCORING_TENSOR and (d % 64 != 0 or k1 > 512)
+
+
 def host_bits(t):
     return synth.bf16_bits(t)
 
@@ -92,24 +102,24 @@ def _workload_case(evk, name, b, n_oracle, stage=0, scoring=None, n=None):
     return wl, mem, q_tab
 
 
-def test_mid_bank_retrieve_and_lognormal_updates(evk):
-    wl, mem, q_tab = _workload_case(evk, "mid", 256, 24, stage=1)
+def test_mid_bank_retrieve_and_lognormal_updates(evk, scoring):
+    wl, mem, q_tab = _workload_case(evk, "mid", 256, 24, stage=1, scoring=scoring)
     ids, r = synth.make_updates(wl)
     evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 1, torch.from_numpy(r).to(DEV), wl.alpha)
     parity.check_update(q_tab[1], ids, r, wl.alpha, evk.evk_q_read(mem, 1).cpu().numpy())
 
 
-def test_clustered_bank(evk):
-    _workload_case(evk, "clustered", 1024, 12)
+def test_clustered_bank(evk, scoring):
+    _workload_case(evk, "clustered", 1024, 12, scoring=scoring)
 
 
 @pytest.mark.parametrize("b", [1, 8, 64])
-def test_large_bank_small_batches(evk, b):
-    _workload_case(evk, "large_hbm", b, 6)
+def test_large_bank_small_batches(evk, b, scoring):
+    _workload_case(evk, "large_hbm", b, 6, scoring=scoring)
 
 
-def test_large_bank_big_batch_with_zipf_updates(evk):
-    wl, mem, q_tab = _workload_case(evk, "large_compute", 4096, 4)
+def test_large_bank_big_batch_with_zipf_updates(evk, scoring):
+    wl, mem, q_tab = _workload_case(evk, "large_compute", 4096, 4, scoring=scoring)
     q = q_tab.copy()
     for rnd in range(3):                       # streaming updates, stage alternating by round
         stage = rnd % 2
@@ -125,11 +135,16 @@ def test_large_bank_big_batch_with_zipf_updates(evk):
 # edge cases
 # ---------------------------------------------------------------------------
 
-def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None):
+def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None, scoring=None):
     bank = synth.gaussian_unit(n, d, seed, DEV)
     queries = synth.gaussian_unit(b, d, seed + 1, DEV)
     q_tab = np.random.default_rng(seed).random((2, max(n, 1))).astype(np.float32)[:, :n]
-    mem = make_mem(evk, bank, np.ascontiguousarray(q_tab), capacity=capacity)
+    mem = make_mem(evk, bank, np.ascontiguousarray(q_tab), capacity=capacity, scoring=scoring)
+    if tensor_unsupported(evk, scoring, d, k1):
+        with pytest.raises(evk.EvkError) as e:
+            evk.evk_retrieve(mem, queries, 0, k1, k2, w)
+        assert e.value.status == evk.EVK_ERR_UNSUPPORTED
+        return mem, None
     out = run_retrieve(evk, mem, queries, 0, k1, k2, w)
     if n:
         ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, k2, w, out)
@@ -144,13 +159,16 @@ def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None):
     (4097, 2048, 2, 1024, 16),   # widest rows, largest pool
     (70001, 256, 9, 33, 5),      # several tiles per block plus a tail
     (20000, 1024, 4, 1, 1),      # k1 = k2 = 1: plain argmax
+    (300, 64, 130, 16, 4),       # two query tiles, the second nearly empty; bank just over one tile
+    (66000, 128, 150, 512, 32),  # sampled thresholds, two query tiles, widest pool of the tensor path
 ])
-def test_edge_shapes(evk, n, d, b, k1, k2):
-    _random_case(evk, n, d, b, k1, k2, 0.5, seed=n)
+def test_edge_shapes(evk, n, d, b, k1, k2, scoring):
+    _random_case(evk, n, d, b, k1, k2, 0.5, seed=n, scoring=scoring)
 
 
-def test_empty_bank_and_empty_batch(evk):
+def test_empty_bank_and_empty_batch(evk, scoring):
     mem = evk.evk_mem_create(64, 128)
+    evk.evk_mem_set_scoring(mem, scoring)
     queries = synth.gaussian_unit(4, 64, 1, DEV)
     ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, 16, 4, 0.5)
     assert np.all(ids == -1) and np.all(np.isneginf(scores))
@@ -162,13 +180,13 @@ def test_empty_bank_and_empty_batch(evk):
     assert evk.evk_last_status(mem) == 0
 
 
-def test_orthonormal_bank_is_exact(evk):
+def test_orthonormal_bank_is_exact(evk, scoring):
     # sims are exact powers of two: no tolerance anywhere
     d = 64
     perm = np.random.default_rng(0).permutation(d)
     bank = torch.eye(d, dtype=torch.float32)[perm].to(DEV)
     q = (2.0 ** -torch.arange(d, dtype=torch.float32))[None, :].to(DEV)
-    mem = make_mem(evk, bank, np.zeros((2, d), np.float32))
+    mem = make_mem(evk, bank, np.zeros((2, d), np.float32), scoring=scoring)
     ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, q, 0, 10, 10, 0.0)
     inv = np.argsort(perm)
     assert pool_ids[0].tolist() == [int(inv[i]) for i in range(10)]
@@ -176,14 +194,14 @@ def test_orthonormal_bank_is_exact(evk):
     assert ids[0].tolist() == pool_ids[0].tolist()
 
 
-def test_ties_break_by_id_and_degenerate_scores(evk):
+def test_ties_break_by_id_and_degenerate_scores(evk, scoring):
     # duplicate rows tie exactly; a zero query makes every similarity equal
     d, n = 128, 3000
     bank = synth.gaussian_unit(n, d, 5, DEV)
     bank[1234] = bank[17]
     bank[2999] = bank[17]
     q_tab = np.zeros((2, n), np.float32)
-    mem = make_mem(evk, bank, q_tab)
+    mem = make_mem(evk, bank, q_tab, scoring=scoring)
     queries = torch.cat([bank[17:18], torch.zeros((1, d), dtype=torch.bfloat16, device=DEV)])
     ids, scores, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, 40, 8, 0.0)
     assert pool_ids[0, :3].tolist() == [17, 1234, 2999]
@@ -193,27 +211,27 @@ def test_ties_break_by_id_and_degenerate_scores(evk):
                           (ids, scores, pool_ids, pool_sims))
 
 
-def test_bank_sorted_against_the_scan(evk):
+@pytest.mark.parametrize("n", [50000, 3000])
+def test_bank_sorted_against_the_scan(evk, scoring, n):
     # similarities increase with the row index, so every row beats the running threshold:
     # the worst case for candidate-list upkeep.
-    d, n = 256, 50000
+    d = 256
     q = synth.gaussian_unit(1, d, 9, DEV)
     bank = synth.gaussian_unit(n, d, 10, DEV)
     sims = (bank.float() @ q.float().T).squeeze(1)
     bank = bank[torch.argsort(sims)].contiguous()
     q_tab = np.random.default_rng(1).random((2, n)).astype(np.float32)
-    mem = make_mem(evk, bank, q_tab)
+    mem = make_mem(evk, bank, q_tab, scoring=scoring)
     out = run_retrieve(evk, mem, q, 1, 256, 16, 0.5)
-    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(q), q_tab[1], 256, 16, 0.5, out)
-    assert ep == 1.0
+    parity.check_retrieve(host_bits(bank), host_bits(q), q_tab[1], 256, 16, 0.5, out)
 
 
-def test_special_weights_and_stage_separation(evk):
+def test_special_weights_and_stage_separation(evk, scoring):
     n, d, b, k1, k2 = 5000, 128, 6, 32, 5
     bank = synth.gaussian_unit(n, d, 21, DEV)
     queries = synth.gaussian_unit(b, d, 22, DEV)
     q_tab = np.random.default_rng(2).random((2, n)).astype(np.float32)
-    mem = make_mem(evk, bank, q_tab)
+    mem = make_mem(evk, bank, q_tab, scoring=scoring)
     ids0, sc0, pool_ids, pool_sims = run_retrieve(evk, mem, queries, 0, k1, k2, 0.0)
     assert np.array_equal(ids0, pool_ids[:, :k2]) and np.array_equal(sc0, pool_sims[:, :k2])
     for stage in (0, 1):
@@ -234,11 +252,11 @@ def test_special_weights_and_stage_separation(evk):
         assert np.array_equal(x, y)
 
 
-def test_fp32_queries_equal_pre_rounded_bf16_queries(evk):
+def test_fp32_queries_equal_pre_rounded_bf16_queries(evk, scoring):
     n, d = 3000, 512
     bank = synth.gaussian_unit(n, d, 31, DEV)
     q32 = synth.gaussian_unit(5, d, 32, DEV, dtype=torch.float32)
-    mem = make_mem(evk, bank, np.zeros((2, n), np.float32))
+    mem = make_mem(evk, bank, np.zeros((2, n), np.float32), scoring=scoring)
     a = run_retrieve(evk, mem, q32, 0, 50, 7, 0.5)
     b = run_retrieve(evk, mem, q32.to(torch.bfloat16), 0, 50, 7, 0.5)
     for x, y in zip(a, b):
@@ -325,12 +343,12 @@ def test_bad_updates_are_rejected_before_any_write(evk):
         evk.evk_retrieve(mem, queries, 2, 8, 2, 0.5)               # stage out of range
 
 
-def test_runs_are_bitwise_repeatable(evk):
+def test_runs_are_bitwise_repeatable(evk, scoring):
     n, d = 40000, 512
     bank = synth.gaussian_unit(n, d, 71, DEV)
     queries = synth.gaussian_unit(11, d, 72, DEV)
     q_tab = np.random.default_rng(4).random((2, n)).astype(np.float32)
-    mem = make_mem(evk, bank, q_tab)
+    mem = make_mem(evk, bank, q_tab, scoring=scoring)
     a = run_retrieve(evk, mem, queries, 0, 128, 8, 0.5)
     for _ in range(3):
         b = run_retrieve(evk, mem, queries, 0, 128, 8, 0.5)
@@ -354,3 +372,58 @@ def test_host_buffer_entry_points(evk):
     r = torch.ones(ids.numel()).pin_memory()
     evk.evk_q_update_host(mem, ids, 0, r, 0.25)
     parity.check_update(q_tab[0], ids.numpy(), r.numpy(), 0.25, evk.evk_q_read(mem, 0).cpu().numpy())
+
+
+def test_both_kernels_return_the_same_pool(evk):
+    # the two phase-1 kernels sum in different orders, so similarities may differ in the last
+    # bits; the id sets agree except where two entries are within rounding of the boundary
+    n, d, b, k1 = 200000, 768, 40, 128
+    bank = synth.gaussian_unit(n, d, 91, DEV)
+    queries = synth.gaussian_unit(b, d, 92, DEV)
+    q_tab = np.random.default_rng(6).random((2, n)).astype(np.float32)
+    outs = []
+    for mode in (evk.EVK_SCORING_STREAM, evk.EVK_SCORING_TENSOR, evk.EVK_SCORING_AUTO):
+        mem = make_mem(evk, bank, q_tab, scoring=mode)
+        kind, launches = evk.evk_retrieve_plan(mem, b, k1)
+        assert kind == (evk.EVK_SCORING_STREAM if mode == evk.EVK_SCORING_STREAM else evk.EVK_SCORING_TENSOR)
+        outs.append(run_retrieve(evk, mem, queries, 0, k1, 8, 0.5))
+    same = sum(set(outs[0][2][i].tolist()) == set(outs[1][2][i].tolist()) for i in range(b))
+    assert same >= b - 2
+    np.testing.assert_allclose(np.sort(outs[0][3], axis=1), np.sort(outs[1][3], axis=1), rtol=1e-4, atol=1e-6)
+    for x, y in zip(outs[1], outs[2]):
+        assert np.array_equal(x, y)
+
+
+def test_sample_rows_recompute_to_the_same_bits(evk):
+    # the starting threshold of the tensor path is a similarity computed in a separate pass over
+    # sampled rows; the scan must reproduce it exactly, or a query could end up short of k1
+    # candidates (the library would then report EVK_ERR_INCOMPLETE)
+    n, d = 120000, 1024
+    bank = synth.gaussian_unit(n, d, 93, DEV)
+    queries = synth.gaussian_unit(133, d, 94, DEV)
+    mem = make_mem(evk, bank, np.zeros((2, n), np.float32), scoring=evk.EVK_SCORING_TENSOR)
+    for k1 in (1, 7, 512):
+        out = evk.evk_retrieve(mem, queries, 0, k1, 1, 0.0, return_pool=True)
+        assert evk.evk_last_status(mem) == 0
+        assert int((out[2] >= 0).sum()) == 133 * k1
+
+
+def test_tensor_path_candidate_lists_overflow_and_are_cut_back(evk):
+    # too small a bank for sampled thresholds and only a few bank splits per query tile: every
+    # row passes the initial threshold, so each query's list fills and is cut back several times
+    n, d, b, k1 = 16000, 64, 2000, 100
+    bank = synth.gaussian_unit(n, d, 95, DEV)
+    queries = synth.gaussian_unit(b, d, 96, DEV)
+    q_tab = np.random.default_rng(8).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    out = run_retrieve(evk, mem, queries, 0, k1, 10, 0.5)
+    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, 10, 0.5, out,
+                                   sample=sample_of(b, 96))
+    assert ep >= 0.9 and ef >= 0.9
+    # and the same with one query whose similarities rise along the scan
+    q1 = queries[:1]
+    order = torch.argsort((bank.float() @ q1.float().T).squeeze(1))
+    bank2 = bank[order].contiguous()
+    mem2 = make_mem(evk, bank2, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    out2 = run_retrieve(evk, mem2, queries, 0, k1, 10, 0.5)
+    parity.check_retrieve(host_bits(bank2), host_bits(queries), q_tab[0], k1, 10, 0.5, out2, sample=[0, 1, 1999])
