@@ -4,9 +4,13 @@
 // B x N similarity matrix of Section 3.2's dense retrieval is never written out.
 //
 // Layout of one thread block (192 threads, one block per SM, persistent):
-//   warp 0     TMA producer: streams 64-column slices of the query tile (A, 128 rows)
-//              and of a bank tile (B, 256 rows) into a 4-stage shared-memory ring,
-//              128-byte swizzled, K-major.
+//   warp 0     TMA producer: streams 64-column slices of a bank tile (B operand, 256
+//              rows) into a shared-memory ring, 128-byte swizzled, K-major.  The query
+//              tile (A operand) is loaded once and stays in shared memory when the
+//              batch is small enough (<= 64 queries of width 1024); otherwise its
+//              slices travel through the ring next to the bank's.  Small batches must
+//              not re-read the queries per bank tile: every block would ask L2 for
+//              the same few lines at the same moment.
 //   warp 1     MMA issuer: one thread issues tcgen05.mma 128x256x16 per 16 columns of
 //              a slice, accumulating D[query][bank row] in one of two 256-column
 //              tensor-memory buffers; tcgen05.commit hands smem stages back to the
@@ -29,6 +33,15 @@
 // strided sample of the bank; its k1-th largest value per query is a safe starting
 // threshold for the full scan (at least k1 entries of the bank reach it).
 //
+// During the full scan the blocks tighten the thresholds together.  Each query has a
+// small histogram in global memory over the similarity range above its starting
+// threshold; every survivor is counted in it, and before each bank tile a thread reads
+// its query's counters and raises its threshold to the highest bin edge that already has
+// k1 survivors at or above it.  Counters only grow, so whatever mix of old and new
+// values a reader sees undercounts, and a threshold derived from it still has at least
+// k1 real entries above it: the selection stays exact while the survivor rate falls
+// from k1/sample to about k1/(rows scanned so far by all blocks).
+//
 // Every wait on an mbarrier is bounded; a wait that runs out raises the block's
 // abort flag, every role leaves its loop, tensor memory is released and the status
 // word reports EVK_ERR_DEVICE_TIMEOUT.
@@ -45,13 +58,14 @@ constexpr int kBlockM = 128;
 constexpr int kBlockN = 256;
 constexpr int kBlockK = 64;
 constexpr int kUmmaK = 16;
-constexpr int kStages = 4;
+constexpr int kMaxStages = 6;
 constexpr int kThreads = 192;
-constexpr uint32_t kABytes = kBlockM * kBlockK * 2;  // 16 KB
-constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;  // 32 KB
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kABytes = kBlockM * kBlockK * 2;  // 16 KB: a streamed slice of the query tile
+constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;  // 32 KB: a slice of a bank tile
 constexpr uint32_t kTmemCols = 512;                  // two accumulators of 256 fp32 columns
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+constexpr size_t kSmemMax = 232448;                  // 227 KB of dynamic shared memory per block
+constexpr size_t kSmemFixed = 1024 + 256;            // alignment slack + barriers
+constexpr int kHistBins = 64;
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
 
 // tcgen05 instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=256, M=128.
@@ -63,7 +77,12 @@ struct MmaParams {
     int B, d, k1;
     int n_qt, splits, n_tiles;
     int mode;           // 0 = filter, 1 = dense
+    int a_resident;     // 1: the query tile is loaded once (n_qt == 1), 0: streamed with the bank
+    int a_rows;         // rows of the query TMA box (multiple of 8)
+    int n_stages;       // depth of the shared-memory ring
     const float *tau0;  // [B] starting thresholds, or nullptr
+    const float2 *range;  // [B] (lowest counted similarity, bins per unit) of the shared histogram
+    unsigned *hist;       // [B][kHistBins] survivors counted by similarity bin
     uint64_t *cand;     // [n_qt*splits][128][kMmaCandCap]
     int *cand_cnt;      // [n_qt*splits][128]
     float *dense;       // [B][dense_ld]
@@ -235,16 +254,26 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     unsigned char *tiles_ptr = smem_raw + (tiles - raw);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tiles_ptr + (size_t)kStages * kStageBytes);
-    // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kStages + 4);
+    const int n_jobs = p.n_qt * p.splits;
+    const int k_chunks = p.d / kBlockK;
+    // [resident query tile: k_chunks slices of a_rows x 128 B] [ring of n_stages stages] [barriers]
+    const uint32_t a_slice = (uint32_t)p.a_rows * 128u;
+    const uint32_t a_region = p.a_resident ? (uint32_t)k_chunks * a_slice : 0u;
+    const uint32_t stage_bytes = p.a_resident ? kBBytes : (kABytes + kBBytes);
+    const uint32_t b_off = p.a_resident ? 0u : kABytes;   // the bank slice inside a stage
+    const uint32_t ring = tiles + a_region;
+    const int kStages = p.n_stages;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tiles_ptr + a_region + (size_t)kStages * stage_bytes);
+    // bars[0..6) full, [6..12) empty, [12..14) tmem_full, [14..16) tmem_empty, [16] queries resident
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 5);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
-    const uint32_t tfull0 = empty0 + 8 * kStages, tempty0 = tfull0 + 16;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
+    const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16, afull = tempty0 + 16;
 
     if (threadIdx.x == 0) {
+        mbar_init(afull, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
@@ -267,24 +296,24 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_jobs = p.n_qt * p.splits;
-    const int k_chunks = p.d / kBlockK;
-
     if (warp == 0) {
         // ===== TMA producer =====
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            if (p.a_resident && blockIdx.x < n_jobs) {
+                mbar_arrive_expect_tx(afull, a_region);
+                for (int kc = 0; kc < k_chunks; ++kc) tma_load_2d(tiles + kc * a_slice, &map_q, afull, kc * kBlockK, 0);
+            }
             for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
                 const int qt = job / p.splits, split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                     for (int kc = 0; kc < k_chunks; ++kc) {
                         if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                        const uint32_t a_dst = tiles + stage * kStageBytes;
-                        const uint32_t b_dst = a_dst + kABytes;
-                        mbar_arrive_expect_tx(full0 + 8 * stage, kStageBytes);
-                        tma_load_2d(a_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
-                        tma_load_2d(b_dst, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
+                        const uint32_t s_dst = ring + stage * stage_bytes;
+                        mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
+                        if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
+                        tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                 }
@@ -295,6 +324,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
+            if (p.a_resident && blockIdx.x < n_jobs) ok = mbar_wait(afull, 0, abort_flag);
             for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
                 const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
@@ -304,9 +334,11 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     for (int kc = 0; kc < k_chunks; ++kc) {
                         if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t a_addr = tiles + stage * kStageBytes;
-                        const uint64_t a_desc = smem_desc(a_addr);
-                        const uint64_t b_desc = smem_desc(a_addr + kABytes);
+                        // a resident query tile narrower than 128 rows is read past its end: the
+                        // surplus accumulator rows belong to no query and are never looked at
+                        const uint32_t s_addr = ring + stage * stage_bytes;
+                        const uint64_t a_desc = smem_desc(p.a_resident ? tiles + kc * a_slice : s_addr);
+                        const uint64_t b_desc = smem_desc(s_addr + b_off);
 #pragma unroll
                         for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
@@ -332,17 +364,28 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int qt = job / p.splits, split = job % p.splits;
             const int q = qt * kBlockM + m;
             const bool q_valid = q < p.B;
-            float tau_sim = INFINITY;
+            // Two filters, both lower bounds of the query's final k1-th key: the key threshold of this
+            // list (exact, rises when the list is cut back) and the bin threshold shared through
+            // the histogram.  tau_sim is a float no larger than either, for the cheap first test.
+            float tau_sim = INFINITY, key_sim_floor = INFINITY;
             uint64_t tau_key = ~(uint64_t)0;
+            float h_lo = 0.0f, h_scale = 0.0f;
+            int tau_bin = 0;
+            unsigned *my_hist = nullptr;
             if (q_valid) {
                 if (p.tau0) {
                     // every entry whose similarity reaches the sampled threshold passes
-                    tau_sim = p.tau0[q];
-                    tau_key = (uint64_t)ordered_bits(tau_sim + 0.0f) << 32;
+                    key_sim_floor = p.tau0[q];
+                    tau_key = (uint64_t)ordered_bits(key_sim_floor + 0.0f) << 32;
+                    const float2 r = p.range[q];
+                    h_lo = r.x;
+                    h_scale = r.y;
+                    if (h_scale > 0.0f) my_hist = p.hist + (size_t)q * kHistBins;
                 } else {
-                    tau_sim = -INFINITY;
+                    key_sim_floor = -INFINITY;
                     tau_key = 0;
                 }
+                tau_sim = key_sim_floor;
             }
             int cnt = 0;
             uint64_t *my_buf = p.cand + ((size_t)job * kBlockM + m) * kMmaCandCap;
@@ -351,6 +394,30 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tc_fence_after();
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
                 const int64_t row0 = (int64_t)t * kBlockN;
+                if (my_hist) {
+                    // highest bin with k1 counted survivors at or above it
+                    int acc_cnt = 0, best = 0;
+                    bool found = false;
+#pragma unroll
+                    for (int g = kHistBins / 4 - 1; g >= 0; --g) {
+                        const uint4 c = __ldcg(reinterpret_cast<const uint4 *>(my_hist) + g);
+                        const unsigned cs[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                        for (int e = 3; e >= 0; --e) {
+                            acc_cnt += (int)cs[e];
+                            if (!found && acc_cnt >= p.k1) {
+                                found = true;
+                                best = g * 4 + e;
+                            }
+                        }
+                    }
+                    if (best > tau_bin) {
+                        tau_bin = best;
+                        // a similarity in bin b is at least h_lo + b / h_scale up to rounding; stay a
+                        // hundredth of a bin below that and let the bin test decide
+                        tau_sim = fmaxf(key_sim_floor, h_lo + ((float)tau_bin - 0.01f) / h_scale);
+                    }
+                }
 #pragma unroll 1
                 for (int c0 = 0; c0 < kBlockN; c0 += 32) {
                     uint32_t v[32];
@@ -375,7 +442,15 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                             const int64_t row = row0 + c0 + j;
                             if (s >= tau_sim && row < p.size) {
                                 const uint64_t key = make_key(s, (int32_t)row);
-                                if (key > tau_key) my_buf[cnt++] = key;
+                                int bin = 0;
+                                if (my_hist) {
+                                    bin = (int)floorf((s - h_lo) * h_scale);
+                                    bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
+                                }
+                                if (key > tau_key && bin >= tau_bin) {
+                                    my_buf[cnt++] = key;
+                                    if (my_hist) atomicAdd(my_hist + bin, 1u);
+                                }
                             }
                         }
                     }
@@ -392,7 +467,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         if (lane == owner) {
                             cnt = p.k1;
                             tau_key = kth;
-                            tau_sim = key_sim(kth);
+                            key_sim_floor = key_sim(kth);
+                            tau_sim = fmaxf(tau_sim, key_sim_floor);
                         }
                     }
                 }
@@ -425,15 +501,31 @@ constexpr int kSelThreads = 512;
 constexpr int kSelPerThread = kMmaSample / kSelThreads;
 
 __global__ void __launch_bounds__(kSelThreads)
-sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0) {
+sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0,
+                        float2 *__restrict__ range, unsigned *__restrict__ hist_out) {
     __shared__ uint64_t keys[kMmaSample];
     __shared__ int hist[256];
     __shared__ uint64_t scal[4];
+    __shared__ unsigned long long top;
     const int q = blockIdx.x;
+    if (threadIdx.x == 0) top = 0;
     for (int i = threadIdx.x; i < n_sample; i += kSelThreads) keys[i] = make_key(dense[(size_t)q * ld + i], i);
+    for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) hist_out[(size_t)q * kHistBins + i] = 0;
     __syncthreads();
     const uint64_t kth = block_select_topk<kSelThreads, kSelPerThread>(keys, n_sample, k1, hist, scal);
-    if (threadIdx.x == 0) tau0[q] = key_sim(kth);
+    for (int i = threadIdx.x; i < k1; i += kSelThreads) atomicMax(&top, (unsigned long long)keys[i]);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // the shared histogram spans from the starting threshold to half a range above the sample's
+        // best similarity; whatever lies higher is counted in the last bin
+        const float lo = key_sim(kth), best = key_sim((uint64_t)top);
+        const float hi = best + 0.5f * (best - lo);
+        float scale = 0.0f;  // 0 switches the histogram off (a sample without spread)
+        if (hi - lo > 1e-2f * fmaxf(fabsf(lo), fabsf(hi)) && hi - lo > 1e-30f) scale = (float)kHistBins / (hi - lo);
+        if (!(scale > 0.0f) || !(scale < 3.0e38f)) scale = 0.0f;
+        tau0[q] = lo;
+        range[q] = make_float2(lo, scale);
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -467,16 +559,42 @@ bool make_map(CUtensorMap *map, const void *base, int d, int64_t rows, int64_t r
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Shared-memory plan for a batch: does the query tile stay resident, how deep is the ring.
+struct SmemPlan {
+    int a_resident, a_rows, n_stages;
+    size_t bytes;
+};
+
+SmemPlan smem_plan(int B, int d) {
+    SmemPlan sp;
+    const int rows = B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM;
+    const size_t a_bytes = (size_t)rows * d * 2;
+    const size_t budget = kSmemMax - kSmemFixed;
+    if (B <= kBlockM && a_bytes + 3 * (size_t)kBBytes <= budget) {
+        sp.a_resident = 1;
+        sp.a_rows = rows;
+        size_t st = (budget - a_bytes) / kBBytes;
+        sp.n_stages = (int)(st > (size_t)kMaxStages ? kMaxStages : st);
+        sp.bytes = kSmemFixed + a_bytes + (size_t)sp.n_stages * kBBytes;
+    } else {
+        sp.a_resident = 0;
+        sp.a_rows = kBlockM;
+        sp.n_stages = 4;
+        sp.bytes = kSmemFixed + (size_t)sp.n_stages * (kABytes + kBBytes);
+    }
+    return sp;
+}
+
 cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
-                          cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+                          size_t smem_bytes, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) return e;
-    score_mma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mq, mb, p);
+    score_mma_kernel<<<grid, kThreads, smem_bytes, stream>>>(mq, mb, p);
     return cudaGetLastError();
 }
 
 struct MmaLayout {
-    size_t cand, cand_cnt, dense, tau0, total;
+    size_t cand, cand_cnt, dense, tau0, range, hist, total;
 };
 
 MmaLayout mma_layout(int B) {
@@ -489,7 +607,9 @@ MmaLayout mma_layout(int B) {
     l.cand_cnt = l.cand + align(lists * kMmaCandCap * sizeof(uint64_t));
     l.dense = l.cand_cnt + align(lists * sizeof(int));
     l.tau0 = l.dense + align(n_qt * kBlockM * kMmaSample * sizeof(float));
-    l.total = l.tau0 + align(n_qt * kBlockM * sizeof(float));
+    l.range = l.tau0 + align(n_qt * kBlockM * sizeof(float));
+    l.hist = l.range + align(n_qt * kBlockM * sizeof(float2));
+    l.total = l.hist + align(n_qt * kBlockM * kHistBins * sizeof(unsigned));
     return l;
 }
 
@@ -532,11 +652,14 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     int *cand_cnt = reinterpret_cast<int *>(ws + l.cand_cnt);
     float *dense = reinterpret_cast<float *>(ws + l.dense);
     float *tau0 = reinterpret_cast<float *>(ws + l.tau0);
+    float2 *range = reinterpret_cast<float2 *>(ws + l.range);
+    unsigned *hist = reinterpret_cast<unsigned *>(ws + l.hist);
     *cand_out = cand;
     *cand_cnt_out = cand_cnt;
 
+    const SmemPlan sp = smem_plan(B, d);
     CUtensorMap map_q, map_bank;
-    if (!make_map(&map_q, queries, d, B, d, kBlockM)) return cudaErrorInvalidValue;
+    if (!make_map(&map_q, queries, d, B, d, sp.a_rows)) return cudaErrorInvalidValue;
 
     MmaParams p;
     p.B = B;
@@ -549,6 +672,11 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.dense_ld = kMmaSample;
     p.status = status;
     p.tau0 = nullptr;
+    p.range = range;
+    p.hist = hist;
+    p.a_resident = sp.a_resident;
+    p.a_rows = sp.a_rows;
+    p.n_stages = sp.n_stages;
 
     if (pl.n_sample) {
         // dense pass over every sample_stride-th row
@@ -559,10 +687,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.n_tiles = pl.n_sample / kBlockN;
         p.splits = splits_for(p.n_qt, p.n_tiles);
         const int jobs = p.n_qt * p.splits;
-        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, stream);
+        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, stream);
         if (err != cudaSuccess) return err;
         ++*launches;
-        sample_threshold_kernel<<<B, kSelThreads, 0, stream>>>(dense, kMmaSample, pl.n_sample, k1, tau0);
+        sample_threshold_kernel<<<B, kSelThreads, 0, stream>>>(dense, kMmaSample, pl.n_sample, k1, tau0, range, hist);
         err = cudaGetLastError();
         if (err != cudaSuccess) return err;
         ++*launches;
@@ -576,7 +704,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.splits = pl.splits;
     cudaError_t err = cudaSuccess;
     if (ev_start) err = cudaEventRecord(ev_start, stream);
-    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, stream);
+    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, sp.bytes, stream);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);
