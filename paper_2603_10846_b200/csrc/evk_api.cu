@@ -51,12 +51,12 @@ int pick_kind(const evk_mem *m, int32_t B, int32_t k1) {
     const bool stream_ok = stream_supported(m->cfg.d);
     if (m->scoring == EVK_SCORING_STREAM) return stream_ok ? EVK_SCORING_STREAM : 0;
     if (m->scoring == EVK_SCORING_TENSOR) return tensor_ok ? EVK_SCORING_TENSOR : 0;
-    if (tensor_ok && B > 4) return EVK_SCORING_TENSOR;
+    if (tensor_ok && B > 1) return EVK_SCORING_TENSOR;  // measured: one query streams as fast without the sampling pass
     return stream_ok ? EVK_SCORING_STREAM : (tensor_ok ? EVK_SCORING_TENSOR : 0);
 }
 
 struct RetrieveLayout {
-    size_t q_bf16, pool_ids, pool_sims, scratch, total;
+    size_t q_bf16, scratch, total;
     size_t part_counts, part_keys;  // streaming kernel only, inside scratch
     int nparts_max;
 };
@@ -65,9 +65,7 @@ RetrieveLayout retrieve_layout(const evk_mem *m, int32_t B, int32_t k1, int kind
     RetrieveLayout l;
     const size_t b = (size_t)(B > 0 ? B : 0);
     l.q_bf16 = 0;
-    l.pool_ids = l.q_bf16 + align256(b * m->cfg.d * sizeof(__nv_bfloat16));
-    l.pool_sims = l.pool_ids + align256(b * k1 * sizeof(int32_t));
-    l.scratch = l.pool_sims + align256(b * k1 * sizeof(float));
+    l.scratch = l.q_bf16 + align256(b * m->cfg.d * sizeof(__nv_bfloat16));
     l.part_counts = l.part_keys = 0;
     l.nparts_max = 0;
     size_t scratch_bytes = 256;
@@ -190,8 +188,6 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
         q_bf16 = dst;
     }
 
-    int32_t *pool_ids = reinterpret_cast<int32_t *>(ws + l.pool_ids);
-    float *pool_sims = reinterpret_cast<float *>(ws + l.pool_sims);
     cudaEvent_t ev_start = mem->prof_start, ev_stop = mem->prof_stop;
     mem->prof_start = mem->prof_stop = nullptr;
 
@@ -227,11 +223,10 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     }
     const int expect = (int)(mem->size < k1 ? mem->size : k1);
     if (err == cudaSuccess)
-        err = launch_merge_pool(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect, mem->status,
-                                pool_ids, pool_sims, pool_ids_out, pool_sims_out, stream, &launches);
-    if (err == cudaSuccess)
-        err = launch_rerank(pool_ids, pool_sims, B, k1, k2, mem->q_tables + (size_t)stage * mem->cfg.capacity,
-                            w, ids_out, scores_out, stream, &launches);
+        err = launch_merge_rerank(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect, mem->status,
+                                  pool_ids_out, pool_sims_out, k2,
+                                  mem->q_tables + (size_t)stage * mem->cfg.capacity, w, ids_out, scores_out,
+                                  stream, &launches);
     mem->launches += launches;
     return cuda_status(err);
 }

@@ -55,20 +55,17 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
                              int32_t *status, uint64_t **cand_out, int **cand_cnt_out,
                              cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream, int *launches);
 
-// ---- phase 1, pool merge ----------------------------------------------------
+// ---- pool merge + phase 2 ------------------------------------------------------
 // List of (query q, part p): (q / qt_size) * (nparts * qt_size) + p * qt_size + q % qt_size.
 // expect: entries every query must at least have (min(k1, size)); fewer sets EVK_ERR_INCOMPLETE.
 constexpr int kMergeMaxParts = 2048;
-cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
-                              int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
-                              int32_t *pool_ids, float *pool_sims,
-                              int32_t *pool_ids_user, float *pool_sims_user,
-                              cudaStream_t stream, int *launches);
-
-// ---- phase 2, rerank --------------------------------------------------------
-cudaError_t launch_rerank(const int32_t *pool_ids, const float *pool_sims, int B, int k1, int k2,
-                          const float *q_stage, float w, int32_t *ids_out, float *scores_out,
-                          cudaStream_t stream, int *launches);
+// Merges each query's lists into its pool (optionally written to pool_*_user, [B][k1]) and
+// runs phase 2 on it: ids_out / scores_out [B][k2].
+cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
+                                int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                                int32_t *pool_ids_user, float *pool_sims_user,
+                                int k2, const float *q_stage, float w, int32_t *ids_out, float *scores_out,
+                                cudaStream_t stream, int *launches);
 
 // ---- Eq. 4 update -----------------------------------------------------------
 size_t q_update_workspace_bytes(int64_t m);

@@ -1,14 +1,17 @@
-// Phase 1, last step: merge the candidate lists that the scoring kernels left per
-// (query, part) into the final pool C(x) of Section 3.2 — the k1 entries of largest
-// similarity, written in (similarity descending, id ascending) order.
+// The end of a retrieval, one thread block per query:
 //
-// One thread block per query.  Candidates stream through a shared-memory buffer
-// that is cut back to its best k1 by an exact radix select whenever it fills; the
-// survivors are then sorted with a bitonic network.  Because keys are totally
-// ordered and distinct, the result does not depend on the order in which the
-// scoring kernels appended candidates.
+//   1. merge the candidate lists that the scoring kernel left per (query, part) into the
+//      pool C(x) of Section 3.2 — the k1 entries of largest similarity, ordered
+//      (similarity descending, id ascending);
+//   2. phase 2: cut the pool down to k2 with the stage's value estimates (rerank.cuh).
+//
+// Candidates stream through a shared-memory buffer that is cut back to its best k1 by
+// an exact radix select whenever it fills; the survivors are sorted with a bitonic
+// network.  Keys are totally ordered and distinct, so the result does not depend on
+// the order in which the scoring kernel appended candidates.
 #include "evk_common.cuh"
 #include "evk_kernels.cuh"
+#include "rerank.cuh"
 
 namespace evk {
 
@@ -18,12 +21,14 @@ constexpr int kThreads = 512;
 constexpr int kSelPerThread = 8;
 constexpr int kCap = kThreads * kSelPerThread;  // 4096 keys = 32 KB
 constexpr int kBatch = 2048;                    // candidates examined between capacity checks
+static_assert(EVK_MAX_K1 * 3 <= kCap, "rerank scratch lives behind the pool in the key buffer");
 
 __global__ void __launch_bounds__(kThreads)
-merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
-                  int part_stride, int qt_size, int k1, int expect, int32_t *__restrict__ status,
-                  int32_t *__restrict__ pool_ids, float *__restrict__ pool_sims,
-                  int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user) {
+merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
+                    int part_stride, int qt_size, int k1, int expect, int32_t *__restrict__ status,
+                    int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user,
+                    int k2, const float *__restrict__ q_stage, float w,
+                    int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
     __shared__ __align__(16) uint64_t keys[kCap];
     __shared__ int offs[kMergeMaxParts + 1];
     __shared__ int hist[256];
@@ -36,24 +41,22 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
     // list of part p: list0 + p * qt_size
     const size_t list0 = (size_t)(q / qt_size) * ((size_t)nparts * qt_size) + (size_t)(q % qt_size);
 
-    // exclusive scan of the part counts (single thread per 8 parts, then serial over chunks:
-    // nparts is at most a few thousand)
     if (tid == 0) {
         count = 0;
         tau = 0;
+        offs[0] = 0;
     }
     for (int p = tid; p < nparts; p += kThreads) offs[p + 1] = part_counts[list0 + (size_t)p * qt_size];
-    if (tid == 0) offs[0] = 0;
     __syncthreads();
     if (tid < 32) {
-        // warp-serial inclusive scan in chunks of 32
+        // inclusive scan of the part counts, 32 at a time
         int carry = 0;
         for (int base = 0; base < nparts; base += 32) {
-            int p = base + tid;
+            const int p = base + tid;
             int v = (p < nparts) ? offs[p + 1] : 0;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                int u = __shfl_up_sync(0xffffffffu, v, off);
+                const int u = __shfl_up_sync(0xffffffffu, v, off);
                 if (tid >= off) v += u;
             }
             if (p < nparts) offs[p + 1] = v + carry;
@@ -101,31 +104,36 @@ merge_pool_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict_
     for (int i = n + tid; i < np2; i += kThreads) keys[i] = 0;
     __syncthreads();
     block_sort_desc<kThreads>(keys, np2);
-    for (int i = tid; i < k1; i += kThreads) {
-        int32_t id = -1;
-        float s = -INFINITY;
-        if (i < n) {
-            id = key_id(keys[i]);
-            s = key_sim(keys[i]);
+    if (pool_ids_user || pool_sims_user) {
+        for (int i = tid; i < k1; i += kThreads) {
+            int32_t id = -1;
+            float s = -INFINITY;
+            if (i < n) {
+                id = key_id(keys[i]);
+                s = key_sim(keys[i]);
+            }
+            if (pool_ids_user) pool_ids_user[(size_t)q * k1 + i] = id;
+            if (pool_sims_user) pool_sims_user[(size_t)q * k1 + i] = s;
         }
-        pool_ids[(size_t)q * k1 + i] = id;
-        pool_sims[(size_t)q * k1 + i] = s;
-        if (pool_ids_user) pool_ids_user[(size_t)q * k1 + i] = id;
-        if (pool_sims_user) pool_sims_user[(size_t)q * k1 + i] = s;
     }
+    // phase 2 on the pool keys[0..n); scratch behind the pool
+    uint64_t *skey = keys + EVK_MAX_K1;
+    int32_t *sid = reinterpret_cast<int32_t *>(keys + 2 * EVK_MAX_K1);
+    rerank_block<kThreads>(keys, n, k2, q_stage, w, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
 }
 
 }  // namespace
 
-cudaError_t launch_merge_pool(const uint64_t *part_keys, const int *part_counts, int nparts,
-                              int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
-                              int32_t *pool_ids, float *pool_sims,
-                              int32_t *pool_ids_user, float *pool_sims_user,
-                              cudaStream_t stream, int *launches) {
+cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
+                                int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                                int32_t *pool_ids_user, float *pool_sims_user,
+                                int k2, const float *q_stage, float w, int32_t *ids_out, float *scores_out,
+                                cudaStream_t stream, int *launches) {
     if (B <= 0) return cudaSuccess;
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
-    merge_pool_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, qt_size, k1, expect,
-                                                  status, pool_ids, pool_sims, pool_ids_user, pool_sims_user);
+    merge_rerank_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, qt_size, k1, expect,
+                                                    status, pool_ids_user, pool_sims_user, k2, q_stage, w, ids_out,
+                                                    scores_out);
     ++*launches;
     return cudaGetLastError();
 }

@@ -190,6 +190,67 @@ apply_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards,
     q_stage[id] = q;
 }
 
+// Small batches (a retrieved context is B*k2 ids) in ONE launch: a single block checks the
+// batch, sorts (id, position) pairs in shared memory and walks each entry's run.  Sorting by
+// the pair keeps every entry's rewards in array order, as the multi-kernel path does.
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallMax = 8192;
+
+__global__ void __launch_bounds__(kSmallThreads)
+small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int m, int n_pow2,
+                    int64_t size, float alpha, float *__restrict__ q_stage, int32_t *__restrict__ status) {
+    extern __shared__ __align__(16) unsigned char small_smem[];
+    uint64_t *keys = reinterpret_cast<uint64_t *>(small_smem);        // [n_pow2] (id << 32) | position
+    float *r = reinterpret_cast<float *>(keys + n_pow2);               // [m]
+    __shared__ int bad_s;
+    const int tid = threadIdx.x;
+    if (tid == 0) bad_s = 0;
+    __syncthreads();
+    int bad = 0;
+    for (int i = tid; i < n_pow2; i += kSmallThreads) {
+        uint64_t key = ~(uint64_t)0;  // padding sorts last
+        if (i < m) {
+            const int32_t id = ids[i];
+            const float rv = rewards[i];
+            if (id < 0 || id >= size) bad |= kFlagRange;
+            if (!(fabsf(rv) <= 3.402823466e38f)) bad |= kFlagNonFinite;
+            key = ((uint64_t)(uint32_t)id << 32) | (uint32_t)i;
+            r[i] = rv;
+        }
+        keys[i] = key;
+    }
+    if (bad) atomicOr(&bad_s, bad);
+    __syncthreads();
+    if (bad_s) {
+        if (tid == 0 && *status == 0) *status = (bad_s & kFlagRange) ? EVK_ERR_RANGE : EVK_ERR_NONFINITE;
+        return;
+    }
+    // bitonic sort, ascending
+    for (int sz = 2; sz <= n_pow2; sz <<= 1) {
+        for (int stride = sz >> 1; stride > 0; stride >>= 1) {
+            for (int t = tid; t < (n_pow2 >> 1); t += kSmallThreads) {
+                const int lo = 2 * t - (t & (stride - 1));
+                const int hi = lo + stride;
+                const bool asc = ((lo & sz) == 0);
+                const uint64_t a = keys[lo], b = keys[hi];
+                if ((a > b) == asc) { keys[lo] = b; keys[hi] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int t = tid; t < m; t += kSmallThreads) {
+        const uint32_t id = (uint32_t)(keys[t] >> 32);
+        if (t > 0 && (uint32_t)(keys[t - 1] >> 32) == id) continue;  // not the head of its run
+        float q = q_stage[id];
+        for (int j = t; j < m && (uint32_t)(keys[j] >> 32) == id; ++j) {
+            const float diff = __fsub_rn(r[(uint32_t)keys[j]], q);
+            const float step = __fmul_rn(alpha, diff);
+            q = __fadd_rn(q, step);
+        }
+        q_stage[id] = q;
+    }
+}
+
 int num_blocks(int64_t m) { return (int)((m + kTile - 1) / kTile); }
 
 struct UpdateLayout {
@@ -218,6 +279,17 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
                             int64_t m, float alpha, int32_t *status, void *workspace,
                             cudaStream_t stream, int *launches) {
     if (m <= 0) return cudaSuccess;
+    if (m <= kSmallMax) {
+        int n_pow2 = 2;
+        while (n_pow2 < m) n_pow2 <<= 1;
+        const size_t smem = (size_t)n_pow2 * sizeof(uint64_t) + (size_t)m * sizeof(float);
+        cudaError_t e = cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(kSmallMax * (sizeof(uint64_t) + sizeof(float))));
+        if (e != cudaSuccess) return e;
+        small_update_kernel<<<1, kSmallThreads, smem, stream>>>(ids, rewards, (int)m, n_pow2, size, alpha, q_stage, status);
+        ++*launches;
+        return cudaGetLastError();
+    }
     const UpdateLayout l = layout_for(m);
     char *ws = static_cast<char *>(workspace);
     int *flags = reinterpret_cast<int *>(ws + l.flags);
