@@ -208,6 +208,14 @@ def run_evk(args):
     rewards_q = torch.from_numpy((rng.random((n_batches, b)) < 0.4).astype(np.float32)).to(dev)
     # one reward per query, shared by the k2 items of its context
     r_sets = [rewards_q[j].repeat_interleave(wl.k2).contiguous() for j in range(n_batches)]
+    # a workload with its own stream of update batches (popularity-skewed ids) uses those
+    own_updates = None
+    if wl.update_ids == "zipf":
+        own_updates = []
+        for j in range(n_batches):
+            u_ids, u_r = synth.make_updates(wl, round_idx=j + 1000 * rank)
+            own_updates.append((torch.from_numpy(u_ids).to(dev), torch.from_numpy(u_r).to(dev)))
+    n_upd = wl.n_updates if own_updates else b * wl.k2
     ids_out = torch.empty((b, wl.k2), dtype=torch.int32, device=dev)
     scores_out = torch.empty((b, wl.k2), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
@@ -230,7 +238,10 @@ def run_evk(args):
         if events is not None:
             evk.evk_mem_profile_scoring(mem, events[0], events[1])
         evk.evk_retrieve(mem, qs, stage, wl.k1, wl.k2, wl.w, out=(ids_out, scores_out))
-        ids_flat, r_flat = gather_updates(ids_out.reshape(-1), r_sets[i % n_batches])
+        if own_updates:
+            ids_flat, r_flat = gather_updates(*own_updates[i % n_batches])
+        else:
+            ids_flat, r_flat = gather_updates(ids_out.reshape(-1), r_sets[i % n_batches])
         evk.evk_q_update(mem, ids_flat, stage, r_flat, wl.alpha)
 
     # ---- device-resident timing ----
@@ -269,12 +280,18 @@ def run_evk(args):
     ids_h = torch.empty((b, wl.k2), dtype=torch.int32).pin_memory()
     sc_h = torch.empty((b, wl.k2), dtype=torch.float32).pin_memory()
     r_h = [r_sets[j % n_batches].cpu().pin_memory() for j in range(4)]
+    upd_h = None
+    if own_updates:
+        upd_h = [(u.cpu().pin_memory(), r.cpu().pin_memory()) for u, r in own_updates[:4]]
     e2e_steps = args.steps
 
     def e2e_step(i):
         stage = i % 2
         evk.evk_retrieve_host(mem, q_host[i % 4], stage, wl.k1, wl.k2, wl.w, ids_h, sc_h)
-        evk.evk_q_update_host(mem, ids_h.reshape(-1), stage, r_h[i % 4], wl.alpha)
+        if upd_h:
+            evk.evk_q_update_host(mem, upd_h[i % len(upd_h)][0], stage, upd_h[i % len(upd_h)][1], wl.alpha)
+        else:
+            evk.evk_q_update_host(mem, ids_h.reshape(-1), stage, r_h[i % 4], wl.alpha)
 
     for i in range(3):
         e2e_step(i)
@@ -306,8 +323,17 @@ def run_evk(args):
         launch_ms = statistics.mean(score_ms) / max(n_score_launches, 1)
         achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
         flops_per_launch = 2.0 * queries_per_launch * size * wl.d
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+        tflops = flops_per_launch / (launch_ms * 1e-3) / 1e12
+        # arithmetic intensity of a scan is `queries_per_launch` flop per byte; the ridge of this
+        # machine sits near 256, beyond it the tensor cores bound the kernel
+        tensor_bound = queries_per_launch >= 256
+        tensor_peak = peaks["bf16_tflops_sustained"] if elapsed_ms / args.steps > 5.0 else peaks["bf16_tflops"]
+        roofline = {"bound": "tensor" if tensor_bound else "hbm",
+                    "achieved": tflops if tensor_bound else achieved,
+                    "peak": tensor_peak if tensor_bound else peaks["hbm_gbs"],
+                    "unit": "TFLOP/s" if tensor_bound else "GB/s",
+                    "frac": (tflops / tensor_peak) if tensor_bound else achieved / peaks["hbm_gbs"],
+                    "traffic": None, "peak_source": peaks["source"], "gbs": achieved,
                     "kernel": "score_stream" if kind == evk.EVK_SCORING_STREAM else "score_mma",
                     "launches_per_step": n_score_launches, "ms_per_launch": launch_ms,
                     "tflops": flops_per_launch / (launch_ms * 1e-3) / 1e12}
@@ -316,13 +342,13 @@ def run_evk(args):
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{wl.name}: N={wl.n}, d={wl.d} bf16, B={b}, k1={wl.k1}, k2={wl.k2}, w={wl.w}; "
-                                   f"step = insert {n_new} + retrieve {b} + update {b * wl.k2 * world}",
+                                   f"step = insert {n_new} + retrieve {b} + update {n_upd * world}",
                        "l2": "inputs larger than L2 (bank %.2f GiB scanned every step)" % (size * wl.d * 2 / 2 ** 30),
                        "parallelism": "replicated bank, queries sharded by rank, update batches all-gathered"
                        if world > 1 else "single GPU"},
             "entries_scanned_per_s": value * size,
             "roofline": roofline,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": b * wl.d * 2 + b * wl.k2 * 8,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": b * wl.d * 2 + n_upd * 8,
                     "d2h_bytes_per_step": b * wl.k2 * 8, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
