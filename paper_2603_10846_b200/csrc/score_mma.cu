@@ -164,8 +164,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// 32 consecutive fp32 columns of this thread's TMEM lane: the load is asynchronous, the
+// registers hold the data only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -176,7 +177,31 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Waits for every outstanding tcgen05.ld of this thread.  The registers are named as in/out
+// operands so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+          "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+          "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+          "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+        :
+        : "memory");
+}
+
+// v[j] for a run-time j without spilling the array: a 5-level select tree.
+__device__ __forceinline__ uint32_t pick32(const uint32_t (&v)[32], int j) {
+    uint32_t a[16], b[8], c[4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = (j & 1) ? v[2 * i + 1] : v[2 * i];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = (j & 2) ? a[2 * i + 1] : a[2 * i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = (j & 4) ? b[2 * i + 1] : b[2 * i];
+    const uint32_t d0 = (j & 8) ? c[1] : c[0], d1 = (j & 8) ? c[3] : c[2];
+    return (j & 16) ? d1 : d0;
 }
 
 // ---- warp-wide exact selection over one candidate list ------------------------
@@ -418,10 +443,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         tau_sim = fmaxf(key_sim_floor, h_lo + ((float)tau_bin - 0.01f) / h_scale);
                     }
                 }
-#pragma unroll 1
-                for (int c0 = 0; c0 < kBlockN; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(t_addr + c0, v);
+                // One 32-column chunk: store it (dense mode) or file the entries that pass the filters.
+                auto process = [&](uint32_t (&v)[32], int c0) {
                     if (p.mode == 1) {
                         if (q_valid) {
                             float4 *dst = reinterpret_cast<float4 *>(p.dense + (size_t)q * p.dense_ld + row0 + c0);
@@ -430,17 +453,21 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
                                                      __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
                         }
-                        continue;
+                        return;
                     }
                     float mx = __uint_as_float(v[0]);
 #pragma unroll
                     for (int j = 1; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
                     if (mx >= tau_sim) {
+                        uint32_t pass = 0;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float s = __uint_as_float(v[j]);
+                        for (int j = 0; j < 32; ++j) pass |= (__uint_as_float(v[j]) >= tau_sim ? 1u : 0u) << j;
+                        while (pass) {
+                            const int j = __ffs(pass) - 1;
+                            pass &= pass - 1;
+                            const float s = __uint_as_float(pick32(v, j));
                             const int64_t row = row0 + c0 + j;
-                            if (s >= tau_sim && row < p.size) {
+                            if (row < p.size) {
                                 const uint64_t key = make_key(s, (int32_t)row);
                                 int bin = 0;
                                 if (my_hist) {
@@ -471,6 +498,19 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                             tau_sim = fmaxf(tau_sim, key_sim_floor);
                         }
                     }
+                };
+                // two register buffers: the next chunk's load is in flight while one is examined
+                uint32_t va[32], vb[32];
+                tmem_ld32_issue(t_addr, va);
+                tmem_ld_wait(va);
+#pragma unroll 1
+                for (int c0 = 0; c0 < kBlockN; c0 += 64) {
+                    tmem_ld32_issue(t_addr + c0 + 32, vb);
+                    process(va, c0);
+                    tmem_ld_wait(vb);
+                    if (c0 + 64 < kBlockN) tmem_ld32_issue(t_addr + c0 + 64, va);
+                    process(vb, c0 + 32);
+                    if (c0 + 64 < kBlockN) tmem_ld_wait(va);
                 }
                 tc_fence_before();
                 __syncwarp();
