@@ -75,13 +75,24 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
                 }
                 scal[0] = prefix | ((uint64_t)digit << shift);
                 scal[1] = (uint64_t)(kk - c);
+                scal[3] = (uint64_t)local[digit & 7];  // keys left in the chosen bin
             }
         }
         __syncthreads();
         prefix = scal[0];
         kk = (int)scal[1];
         mask |= (uint64_t)0xff << shift;
+        const bool last_one = (scal[3] == 1);
         __syncthreads();
+        if (last_one) {
+            // a single key is left under this prefix: it is the k-th largest
+            for (int i = tid; i < n; i += NT)
+                if ((keys[i] & mask) == prefix) scal[0] = keys[i];
+            __syncthreads();
+            prefix = scal[0];
+            __syncthreads();
+            break;
+        }
     }
     // prefix is now the k-th largest key; exactly k keys are >= prefix.
     uint64_t mine[PER_THREAD];

@@ -100,11 +100,12 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
         block_select_topk<kThreads, kSelPerThread>(keys, n, k1, hist, scal);
         n = k1;
     }
-    const int np2 = next_pow2(n > 1 ? n : 1);
-    for (int i = n + tid; i < np2; i += kThreads) keys[i] = 0;
-    __syncthreads();
-    block_sort_desc<kThreads>(keys, np2);
     if (pool_ids_user || pool_sims_user) {
+        // the pool itself is wanted: put it in (similarity descending, id ascending) order
+        const int np2 = next_pow2(n > 1 ? n : 1);
+        for (int i = n + tid; i < np2; i += kThreads) keys[i] = 0;
+        __syncthreads();
+        block_sort_desc<kThreads>(keys, np2);
         for (int i = tid; i < k1; i += kThreads) {
             int32_t id = -1;
             float s = -INFINITY;
@@ -116,7 +117,8 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
             if (pool_sims_user) pool_sims_user[(size_t)q * k1 + i] = s;
         }
     }
-    // phase 2 on the pool keys[0..n); scratch behind the pool
+    __syncthreads();
+    // phase 2 on the pool keys[0..n) (any order); scratch behind the pool
     uint64_t *skey = keys + EVK_MAX_K1;
     int32_t *sid = reinterpret_cast<int32_t *>(keys + 2 * EVK_MAX_K1);
     rerank_block<kThreads>(keys, n, k2, q_stage, w, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);

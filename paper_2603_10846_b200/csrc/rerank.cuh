@@ -16,7 +16,7 @@ __device__ __forceinline__ bool rerank_before(uint64_t ka, int32_t ia, uint64_t 
     return ka > kb || (ka == kb && (uint32_t)ia < (uint32_t)ib);
 }
 
-// Block-wide: the pool of one query is n sorted keys (sim desc, id asc) in shared memory.
+// Block-wide: the pool of one query is n keys in shared memory, in any order.
 // Gathers Q_stage, scores, sorts, writes the first k2 results (padding: id -1, score -inf).
 // skey / sid: shared scratch of next_pow2(n) entries each.
 template <int NT>

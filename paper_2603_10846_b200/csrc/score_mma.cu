@@ -204,6 +204,13 @@ __device__ __forceinline__ uint32_t pick32(const uint32_t (&v)[32], int j) {
     return (j & 16) ? d1 : d0;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor still runs; pdl_wait blocks until the predecessor has finished
+// and its writes are visible (a no-op in an ordinary launch), pdl_trigger lets the successor
+// start early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- warp-wide exact selection over one candidate list ------------------------
 // The whole warp cuts the list `buf` (n <= kMmaCandCap distinct non-zero keys) back to
 // its k largest and returns the k-th largest key.  Keys live in registers (32 per
@@ -294,6 +301,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_trigger();
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
     const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16, afull = tempty0 + 16;
 
@@ -381,6 +389,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else {
         // ===== epilogue: thread = one query of the tile = one TMEM lane =====
+        // The thresholds, the histogram and the candidate lists belong to the kernels before this
+        // one; loads and MMAs of the first tiles run ahead while the epilogue waits for them.
+        pdl_wait();
         const int quarter = warp & 3;              // warps 2,3,4,5 -> lane quarters 2,3,0,1
         const int m = quarter * 32 + lane;
         uint32_t acc = 0, acc_phase = 0;
@@ -548,6 +559,8 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
     __shared__ uint64_t scal[4];
     __shared__ unsigned long long top;
     const int q = blockIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (threadIdx.x == 0) top = 0;
     for (int i = threadIdx.x; i < n_sample; i += kSelThreads) keys[i] = make_key(dense[(size_t)q * ld + i], i);
     for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) hist_out[(size_t)q * kHistBins + i] = 0;
@@ -625,12 +638,22 @@ SmemPlan smem_plan(int B, int d) {
     return sp;
 }
 
+// overlap = true: programmatic dependent launch behind the kernel enqueued just before.
 cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
-                          size_t smem_bytes, cudaStream_t stream) {
+                          size_t smem_bytes, bool overlap, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) return e;
-    score_mma_kernel<<<grid, kThreads, smem_bytes, stream>>>(mq, mb, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, score_mma_kernel, mq, mb, p);
 }
 
 struct MmaLayout {
@@ -727,11 +750,22 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.n_tiles = pl.n_sample / kBlockN;
         p.splits = splits_for(p.n_qt, p.n_tiles);
         const int jobs = p.n_qt * p.splits;
-        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, stream);
+        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, false, stream);
         if (err != cudaSuccess) return err;
         ++*launches;
-        sample_threshold_kernel<<<B, kSelThreads, 0, stream>>>(dense, kMmaSample, pl.n_sample, k1, tau0, range, hist);
-        err = cudaGetLastError();
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(B);
+            cfg.blockDim = dim3(kSelThreads);
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            err = cudaLaunchKernelEx(&cfg, sample_threshold_kernel, (const float *)dense, (int)kMmaSample,
+                                     (int)pl.n_sample, (int)k1, tau0, range, hist);
+        }
         if (err != cudaSuccess) return err;
         ++*launches;
         p.tau0 = tau0;
@@ -744,7 +778,8 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.splits = pl.splits;
     cudaError_t err = cudaSuccess;
     if (ev_start) err = cudaEventRecord(ev_start, stream);
-    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, sp.bytes, stream);
+    // behind the threshold kernel the scan may start early; its epilogue waits for the thresholds
+    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, sp.bytes, pl.n_sample != 0 && !ev_start, stream);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);
