@@ -131,6 +131,31 @@ __device__ void block_sort_desc(uint64_t *keys, int n_pow2) {
     __syncthreads();
 }
 
+// Programmatic dependent launch.  A kernel launched through launch_overlapped may be scheduled
+// while the kernel enqueued before it on the stream is still running; it must call pdl_wait()
+// before it touches anything an earlier kernel wrote or reads anything it will overwrite.
+// pdl_wait() returns once the preceding kernel has finished and its writes are visible (at
+// once in an ordinary launch).  pdl_trigger() in the earlier kernel lets the next one be
+// scheduled from that point on instead of at the earlier kernel's end.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __host__ __device__ __forceinline__ int next_pow2(int x) {
     int p = 1;
     while (p < x) p <<= 1;

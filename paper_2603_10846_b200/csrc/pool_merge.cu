@@ -38,6 +38,8 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
 
     const int tid = threadIdx.x;
     const int q = blockIdx.x;
+    pdl_trigger();
+    pdl_wait();  // the candidate lists are the scoring kernel's output
     // list of part p: list0 + p * qt_size
     const size_t list0 = (size_t)(q / qt_size) * ((size_t)nparts * qt_size) + (size_t)(q % qt_size);
 
@@ -133,11 +135,10 @@ cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_count
                                 cudaStream_t stream, int *launches) {
     if (B <= 0) return cudaSuccess;
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
-    merge_rerank_kernel<<<B, kThreads, 0, stream>>>(part_keys, part_counts, nparts, part_stride, qt_size, k1, expect,
-                                                    status, pool_ids_user, pool_sims_user, k2, q_stage, w, ids_out,
-                                                    scores_out);
     ++*launches;
-    return cudaGetLastError();
+    return launch_overlapped(merge_rerank_kernel, dim3(B), dim3(kThreads), 0, stream, part_keys, part_counts, nparts,
+                             part_stride, qt_size, k1, expect, status, pool_ids_user, pool_sims_user, k2, q_stage, w,
+                             ids_out, scores_out);
 }
 
 }  // namespace evk

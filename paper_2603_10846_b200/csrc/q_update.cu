@@ -204,6 +204,8 @@ small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ r
     float *r = reinterpret_cast<float *>(keys + n_pow2);               // [m]
     __shared__ int bad_s;
     const int tid = threadIdx.x;
+    pdl_trigger();
+    pdl_wait();  // ids usually come straight out of the retrieval enqueued before
     if (tid == 0) bad_s = 0;
     __syncthreads();
     int bad = 0;
@@ -286,9 +288,9 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
         cudaError_t e = cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kSmallMax * (sizeof(uint64_t) + sizeof(float))));
         if (e != cudaSuccess) return e;
-        small_update_kernel<<<1, kSmallThreads, smem, stream>>>(ids, rewards, (int)m, n_pow2, size, alpha, q_stage, status);
         ++*launches;
-        return cudaGetLastError();
+        return launch_overlapped(small_update_kernel, dim3(1), dim3(kSmallThreads), smem, stream, ids, rewards, (int)m,
+                                 n_pow2, size, alpha, q_stage, status);
     }
     const UpdateLayout l = layout_for(m);
     char *ws = static_cast<char *>(workspace);

@@ -204,13 +204,6 @@ __device__ __forceinline__ uint32_t pick32(const uint32_t (&v)[32], int j) {
     return (j & 16) ? d1 : d0;
 }
 
-// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
-// start while its predecessor still runs; pdl_wait blocks until the predecessor has finished
-// and its writes are visible (a no-op in an ordinary launch), pdl_trigger lets the successor
-// start early.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
 // ---- warp-wide exact selection over one candidate list ------------------------
 // The whole warp cuts the list `buf` (n <= kMmaCandCap distinct non-zero keys) back to
 // its k largest and returns the k-th largest key.  Keys live in registers (32 per
