@@ -175,7 +175,7 @@ def run_reference(args):
 def run_evk(args):
     import torch
     import torch.distributed as dist
-    from paper_2603_10846_b200 import evk, synth
+    from paper_2603_10846_b200 import evk, parallel, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -222,13 +222,7 @@ def run_evk(args):
 
     def gather_updates(ids_flat, rewards_flat):
         """Replicas stay identical: every rank applies every rank's updates, in rank order."""
-        if world == 1:
-            return ids_flat, rewards_flat
-        all_ids = torch.empty(world * ids_flat.numel(), dtype=ids_flat.dtype, device=dev)
-        all_r = torch.empty(world * rewards_flat.numel(), dtype=rewards_flat.dtype, device=dev)
-        dist.all_gather_into_tensor(all_ids, ids_flat)
-        dist.all_gather_into_tensor(all_r, rewards_flat)
-        return all_ids, all_r
+        return parallel.gather_update_batches(ids_flat, rewards_flat)
 
     def step(i, events=None):
         stage = i % 2
