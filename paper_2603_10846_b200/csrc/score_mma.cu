@@ -649,6 +649,29 @@ cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const Mm
     return cudaLaunchKernelEx(&cfg, score_mma_kernel, mq, mb, p);
 }
 
+// Bank splits per query tile.  Jobs (query tile, split) are dealt round-robin to the
+// blocks, one block per SM; the split count is the smallest one from 148 / n_qt upwards whose
+// job count fills whole rounds of 148 blocks to 97 % or better.  Fewer splits keep more query
+// tiles side by side on the same bank tiles (they share them through L2).
+int splits_for(int n_qt, int n_tiles) {
+    if (n_qt <= 0) n_qt = 1;
+    int base = kNumSM / n_qt;
+    if (base < 1) base = 1;
+    int splits = base;
+    if (n_qt < kNumSM) {
+        for (int s = base; s <= 4 * base && s <= kNumSM; ++s) {
+            const int jobs = n_qt * s;
+            const int rounds = (jobs + kNumSM - 1) / kNumSM;
+            if (jobs * 100 >= 97 * rounds * kNumSM) {
+                splits = s;
+                break;
+            }
+        }
+    }
+    if (splits > n_tiles) splits = n_tiles > 0 ? n_tiles : 1;
+    return splits;
+}
+
 struct MmaLayout {
     size_t cand, cand_cnt, dense, tau0, range, hist, total;
 };
@@ -656,8 +679,8 @@ struct MmaLayout {
 MmaLayout mma_layout(int B) {
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t n_qt = (size_t)((B + kBlockM - 1) / kBlockM);
-    // jobs = n_qt * floor(148 / n_qt) <= 148 while n_qt <= 148, else one split per query tile
-    const size_t lists = (n_qt > (size_t)kNumSM ? n_qt : (size_t)kNumSM) * kBlockM;
+    // one candidate list per (job, query of the tile); the split count can only shrink for small banks
+    const size_t lists = n_qt * (size_t)splits_for((int)n_qt, 1 << 30) * kBlockM;
     MmaLayout l;
     l.cand = 0;
     l.cand_cnt = l.cand + align(lists * kMmaCandCap * sizeof(uint64_t));
@@ -667,13 +690,6 @@ MmaLayout mma_layout(int B) {
     l.hist = l.range + align(n_qt * kBlockM * sizeof(float2));
     l.total = l.hist + align(n_qt * kBlockM * kHistBins * sizeof(unsigned));
     return l;
-}
-
-int splits_for(int n_qt, int n_tiles) {
-    int splits = kNumSM / (n_qt > 0 ? n_qt : 1);
-    if (splits < 1) splits = 1;
-    if (splits > n_tiles) splits = n_tiles > 0 ? n_tiles : 1;
-    return splits;
 }
 
 }  // namespace
