@@ -33,6 +33,17 @@ __device__ __forceinline__ uint64_t make_key(float sim, int32_t id) {
 __device__ __forceinline__ float key_sim(uint64_t key) { return from_ordered_bits((uint32_t)(key >> 32)); }
 __device__ __forceinline__ int32_t key_id(uint64_t key) { return (int32_t)(~(uint32_t)key); }
 
+// Claims one slot of a shared counter for every lane whose `want` is set, with a single atomic
+// per warp.  Every lane of the warp must call it; returns the lane's slot (undefined if !want).
+__device__ __forceinline__ int warp_claim_slot(bool want, int *counter) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t votes = __ballot_sync(0xffffffffu, want);
+    int base = 0;
+    if (votes && lane == (uint32_t)(__ffs(votes) - 1)) base = atomicAdd(counter, __popc(votes));
+    base = __shfl_sync(0xffffffffu, base, votes ? (__ffs(votes) - 1) : 0);
+    return base + __popc(votes & ((1u << lane) - 1u));
+}
+
 // ---------------------------------------------------------------------------
 // Block-wide exact selection.  Keeps the k largest of n distinct 64-bit keys held
 // in shared memory and moves them to keys[0..k) (in no particular order).
@@ -50,7 +61,7 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
         for (int i = tid; i < 256; i += NT) hist[i] = 0;
         __syncthreads();
         for (int i = tid; i < n; i += NT) {
-            uint64_t key = keys[i];
+            const uint64_t key = keys[i];
             if ((key & mask) == prefix) atomicAdd(&hist[(int)((key >> shift) & 0xff)], 1);
         }
         __syncthreads();
@@ -106,8 +117,10 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
     __syncthreads();
 #pragma unroll
     for (int j = 0; j < PER_THREAD; ++j) {
-        int i = tid + j * NT;
-        if (i < n && mine[j] >= prefix) keys[atomicAdd(counter, 1)] = mine[j];
+        const int i = tid + j * NT;
+        const bool keep = i < n && mine[j] >= prefix;
+        const int slot = warp_claim_slot(keep, counter);
+        if (keep) keys[slot] = mine[j];
     }
     __syncthreads();
     return prefix;

@@ -73,6 +73,7 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
 #pragma unroll
         for (int j = 0; j < kBatch / kThreads; ++j) {
             const int idx = base + tid + j * kThreads;
+            uint64_t key = 0;
             if (idx < total) {
                 // part p with offs[p] <= idx < offs[p+1]
                 int lo = 0, hi = nparts;
@@ -80,9 +81,11 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
                     const int mid = (lo + hi) >> 1;
                     if (offs[mid] <= idx) lo = mid; else hi = mid;
                 }
-                const uint64_t key = part_keys[(list0 + (size_t)lo * qt_size) * part_stride + (idx - offs[lo])];
-                if (key > t) keys[atomicAdd(&count, 1)] = key;
+                key = part_keys[(list0 + (size_t)lo * qt_size) * part_stride + (idx - offs[lo])];
             }
+            const bool keep = idx < total && key > t;
+            const int slot = warp_claim_slot(keep, &count);
+            if (keep) keys[slot] = key;
         }
         __syncthreads();
         const int n = count;
