@@ -427,3 +427,16 @@ def test_tensor_path_candidate_lists_overflow_and_are_cut_back(evk):
     mem2 = make_mem(evk, bank2, q_tab, scoring=evk.EVK_SCORING_TENSOR)
     out2 = run_retrieve(evk, mem2, queries, 0, k1, 10, 0.5)
     parity.check_retrieve(host_bits(bank2), host_bits(queries), q_tab[0], k1, 10, 0.5, out2, sample=[0, 1, 1999])
+
+
+def test_more_query_tiles_than_sms(evk):
+    # 149 query tiles: each gets a single bank split and blocks take several jobs in turn
+    n, d, b, k1 = 3000, 64, 149 * 128 - 5, 20
+    bank = synth.gaussian_unit(n, d, 97, DEV)
+    queries = synth.gaussian_unit(b, d, 98, DEV)
+    q_tab = np.random.default_rng(9).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    out = run_retrieve(evk, mem, queries, 1, k1, 5, 0.5)
+    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[1], k1, 5, 0.5, out,
+                                   sample=[0, 127, 128, 9000, b - 1] + sample_of(b, 40, seed=3))
+    assert ep >= 0.9 and ef >= 0.9
