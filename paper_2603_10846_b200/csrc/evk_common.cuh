@@ -57,7 +57,38 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
     const int tid = threadIdx.x;
     uint64_t prefix = 0, mask = 0;
     int kk = k;
+    // Bits on which all keys agree (sign and exponent of similarities in a narrow range, the
+    // upper id bits of a small bank) need no pass: every key would fall into one bin, and the
+    // shared-memory atomics on that single counter would run one after another.
+    if (tid < 4) hist[tid] = (tid < 2) ? -1 : 0;  // and_lo, and_hi, or_lo, or_hi
+    __syncthreads();
+    {
+        uint64_t all_and = ~(uint64_t)0, all_or = 0;
+        for (int i = tid; i < n; i += NT) {
+            all_and &= keys[i];
+            all_or |= keys[i];
+        }
+        const uint32_t a_lo = __reduce_and_sync(0xffffffffu, (uint32_t)all_and);
+        const uint32_t a_hi = __reduce_and_sync(0xffffffffu, (uint32_t)(all_and >> 32));
+        const uint32_t o_lo = __reduce_or_sync(0xffffffffu, (uint32_t)all_or);
+        const uint32_t o_hi = __reduce_or_sync(0xffffffffu, (uint32_t)(all_or >> 32));
+        if ((tid & 31) == 0) {
+            atomicAnd(&hist[0], (int)a_lo);
+            atomicAnd(&hist[1], (int)a_hi);
+            atomicOr(&hist[2], (int)o_lo);
+            atomicOr(&hist[3], (int)o_hi);
+        }
+    }
+    __syncthreads();
+    const uint64_t common = ((uint64_t)(uint32_t)hist[1] << 32) | (uint32_t)hist[0];
+    const uint64_t varying = common ^ (((uint64_t)(uint32_t)hist[3] << 32) | (uint32_t)hist[2]);
+    __syncthreads();
     for (int shift = 56; shift >= 0; shift -= 8) {
+        if (((varying >> shift) & 0xff) == 0) {
+            prefix |= common & ((uint64_t)0xff << shift);
+            mask |= (uint64_t)0xff << shift;
+            continue;
+        }
         for (int i = tid; i < 256; i += NT) hist[i] = 0;
         __syncthreads();
         for (int i = tid; i < n; i += NT) {
@@ -129,9 +160,14 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
 // Block-wide bitonic sort of n_pow2 keys in shared memory, descending.
 template <int NT>
 __device__ void block_sort_desc(uint64_t *keys, int n_pow2) {
+    // A stage with stride <= 32 stays inside the 64 elements a warp owns, so a warp sync is
+    // enough between two such stages.
+    bool wide_before = true;
     for (int size = 2; size <= n_pow2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
+            const bool wide = stride > 32;
+            if (wide || wide_before) __syncthreads(); else __syncwarp();
+            wide_before = wide;
             for (int t = threadIdx.x; t < (n_pow2 >> 1); t += NT) {
                 int lo = 2 * t - (t & (stride - 1));
                 int hi = lo + stride;

@@ -228,8 +228,13 @@ small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ r
         return;
     }
     // bitonic sort, ascending
+    // (a stage with stride <= 32 stays inside the 64 elements a warp owns: warp sync is enough)
+    bool wide_before = true;
     for (int sz = 2; sz <= n_pow2; sz <<= 1) {
         for (int stride = sz >> 1; stride > 0; stride >>= 1) {
+            const bool wide = stride > 32;
+            if (wide || wide_before) __syncthreads(); else __syncwarp();
+            wide_before = wide;
             for (int t = tid; t < (n_pow2 >> 1); t += kSmallThreads) {
                 const int lo = 2 * t - (t & (stride - 1));
                 const int hi = lo + stride;
@@ -237,9 +242,9 @@ small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ r
                 const uint64_t a = keys[lo], b = keys[hi];
                 if ((a > b) == asc) { keys[lo] = b; keys[hi] = a; }
             }
-            __syncthreads();
         }
     }
+    __syncthreads();
     for (int t = tid; t < m; t += kSmallThreads) {
         const uint32_t id = (uint32_t)(keys[t] >> 32);
         if (t > 0 && (uint32_t)(keys[t - 1] >> 32) == id) continue;  // not the head of its run

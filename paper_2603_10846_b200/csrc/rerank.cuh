@@ -39,9 +39,12 @@ __device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const flo
         skey[i] = key;
         sid[i] = id;
     }
+    bool wide_before = true;  // stages with stride <= 32 stay inside a warp's own 64 elements
     for (int size = 2; size <= np2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
+            const bool wide = stride > 32;
+            if (wide || wide_before) __syncthreads(); else __syncwarp();
+            wide_before = wide;
             for (int t = tid; t < (np2 >> 1); t += NT) {
                 const int lo = 2 * t - (t & (stride - 1));
                 const int hi = lo + stride;
