@@ -60,6 +60,12 @@ def _load():
     lib.evk_oracle_q_update_f64.restype = None
     lib.evk_oracle_q_update_f32.argtypes = [p, p, p, c_i64, c_f32]
     lib.evk_oracle_q_update_f32.restype = None
+    lib.evk_oracle_reward_draft.argtypes = [p, c_i64, p]
+    lib.evk_oracle_reward_draft.restype = None
+    lib.evk_oracle_reward_refine.argtypes = [p, p, p, c_i64, p]
+    lib.evk_oracle_reward_refine.restype = None
+    lib.evk_oracle_reward_normalize.argtypes = [p, c_i64, p, c_i64, c_f64, c_f64, p]
+    lib.evk_oracle_reward_normalize.restype = None
     _lib = lib
     return lib
 
@@ -169,3 +175,31 @@ def q_update_f32(q_stage, ids, rewards, alpha) -> np.ndarray:
     _load().evk_oracle_q_update_f32(_ptr(q), _ptr(ids), _ptr(rewards), ids.size,
                                     float(np.float32(alpha)))
     return q
+
+
+def reward_draft(feasible) -> np.ndarray:
+    """Eq. 5: +1 if feasible else -1 (fp64)."""
+    f = _c(feasible, np.uint8)
+    out = np.empty(f.shape, dtype=np.float64)
+    _load().evk_oracle_reward_draft(_ptr(f), f.size, _ptr(out))
+    return out
+
+
+def reward_refine(best_latency, latency, feasible) -> np.ndarray:
+    """Eq. 6: -1 if infeasible else tanh(log b - log l) (fp64)."""
+    b = _c(best_latency, np.float32)
+    l = _c(latency, np.float32)
+    f = _c(feasible, np.uint8)
+    assert b.shape == l.shape == f.shape
+    out = np.empty(b.shape, dtype=np.float64)
+    _load().evk_oracle_reward_refine(_ptr(b), _ptr(l), _ptr(f), b.size, _ptr(out))
+    return out
+
+
+def reward_normalize(history, raw, sigma_min: float, clip: float = 0.0) -> np.ndarray:
+    """Running z-score with the statistics of everything seen before each reward."""
+    h = _c(history, np.float64)
+    r = _c(raw, np.float32)
+    out = np.empty(r.shape, dtype=np.float64)
+    _load().evk_oracle_reward_normalize(_ptr(h), h.size, _ptr(r), r.size, float(sigma_min), float(clip), _ptr(out))
+    return out

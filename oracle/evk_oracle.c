@@ -172,3 +172,48 @@ void evk_oracle_q_update_f32(float *q_stage, const int32_t *ids, const float *re
         q_stage[ids[t]] = next;
     }
 }
+
+/* ---- Rewards (Eq. 5, Eq. 6) and their online normalisation (Appendix A) --------- */
+
+/* Eq. 5: the drafting reward is +1 for a feasible kernel and -1 otherwise. */
+void evk_oracle_reward_draft(const uint8_t *feasible, int64_t n, double *out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = feasible[i] ? 1.0 : -1.0;
+}
+
+/* Eq. 6: -1 for an infeasible kernel, otherwise tanh(log b - log l) with b the best
+ * latency so far and l the new one (the speed-up ratio rho = b / l enters as
+ * tanh(log rho), Appendix A "Reward definitions by stage"). */
+void evk_oracle_reward_refine(const float *best, const float *latency, const uint8_t *feasible,
+                              int64_t n, double *out) {
+    for (int64_t i = 0; i < n; ++i)
+        out[i] = feasible[i] ? tanh(log((double)best[i]) - log((double)latency[i])) : -1.0;
+}
+
+/* Running z-score of the raw rewards (Appendix A, "Stability of Online Normalization"):
+ *   R_t = (r_t - mu_{t-1}) / max(sigma_{t-1}, sigma_min),   optionally clipped to [-clip, clip],
+ * with mu_t the mean and sigma_t the POPULATION standard deviation of r_1..r_t, both
+ * recomputed here from their definitions for every t (quadratic work: small inputs only).
+ * history[0..n_hist) are the raw rewards of earlier calls.  While fewer than two rewards
+ * have been seen the raw reward passes through unchanged.  clip <= 0 disables clipping. */
+void evk_oracle_reward_normalize(const double *history, int64_t n_hist, const float *raw, int64_t n,
+                                 double sigma_min, double clip, double *out) {
+    for (int64_t t = 0; t < n; ++t) {
+        const int64_t seen = n_hist + t;
+        double r = (double)raw[t];
+        if (seen >= 2) {
+            double mu = 0.0;
+            for (int64_t k = 0; k < seen; ++k) mu += (k < n_hist) ? history[k] : (double)raw[k - n_hist];
+            mu /= (double)seen;
+            double var = 0.0;
+            for (int64_t k = 0; k < seen; ++k) {
+                const double v = ((k < n_hist) ? history[k] : (double)raw[k - n_hist]) - mu;
+                var += v * v;
+            }
+            double sigma = sqrt(var / (double)seen);
+            if (sigma < sigma_min) sigma = sigma_min;
+            r = (r - mu) / sigma;
+        }
+        if (clip > 0.0) r = r > clip ? clip : (r < -clip ? -clip : r);
+        out[t] = r;
+    }
+}
