@@ -196,6 +196,27 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
                       const float *rewards_host, float alpha,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* Rewards for evk_q_update.  All arrays are device arrays of n elements.
+ *
+ * evk_reward_draft (Eq. 5): +1 where feasible[i] != 0, else -1.
+ * evk_reward_refine (Eq. 6): -1 where infeasible, else tanh(log best_latency[i] - log latency[i])
+ *   (best_latency = the best latency seen before this attempt; latencies must be > 0).
+ * evk_reward_normalize (Appendix A, running normalisation): replaces raw reward r_t by
+ *   (r_t - mu_{t-1}) / max(sigma_{t-1}, sigma_min), clipped to [-clip, clip] if clip > 0, where
+ *   mu and sigma are the mean and population standard deviation of every raw reward that went
+ *   through `state` before r_t (earlier calls and earlier elements of this call, in array
+ *   order).  The first two rewards ever seen pass through unchanged.  Stored values are not
+ *   rescaled when the statistics move.  `state` is evk_reward_norm_state_bytes() bytes of
+ *   device memory, 8-byte aligned, owned by the caller, zeroed by evk_reward_norm_reset; calls
+ *   sharing a state must be ordered on one stream.  sigma_min > 0, clip >= 0 (0 = no clipping). */
+int evk_reward_draft(const uint8_t *feasible, int64_t n, float *rewards_out, void *stream);
+int evk_reward_refine(const float *best_latency, const float *latency, const uint8_t *feasible, int64_t n,
+                      float *rewards_out, void *stream);
+size_t evk_reward_norm_state_bytes(void);
+int evk_reward_norm_reset(void *state, void *stream);
+int evk_reward_normalize(void *state, const float *raw, int64_t n, float sigma_min, float clip,
+                         float *rewards_out, void *stream);
+
 /* What evk_retrieve would run for a batch of B queries at the current size: the
  * phase-1 kernel (EVK_SCORING_STREAM or EVK_SCORING_TENSOR) and how many times it
  * is launched (each launch scans the whole bank once). */

@@ -383,6 +383,40 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
     return cuda_status(cudaStreamSynchronize(stream));
 }
 
+// ---- rewards -------------------------------------------------------------------
+
+int evk_reward_draft(const uint8_t *feasible, int64_t n, float *rewards_out, void *stream) {
+    if (n < 0) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!feasible || !rewards_out) return EVK_ERR_INVALID;
+    return cuda_status(launch_reward_draft(feasible, n, rewards_out, static_cast<cudaStream_t>(stream)));
+}
+
+int evk_reward_refine(const float *best_latency, const float *latency, const uint8_t *feasible, int64_t n,
+                      float *rewards_out, void *stream) {
+    if (n < 0) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!best_latency || !latency || !feasible || !rewards_out) return EVK_ERR_INVALID;
+    return cuda_status(launch_reward_refine(best_latency, latency, feasible, n, rewards_out,
+                                            static_cast<cudaStream_t>(stream)));
+}
+
+size_t evk_reward_norm_state_bytes(void) { return 4 * sizeof(double); }
+
+int evk_reward_norm_reset(void *state, void *stream) {
+    if (!state || !aligned(state, 8)) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemsetAsync(state, 0, evk_reward_norm_state_bytes(), static_cast<cudaStream_t>(stream)));
+}
+
+int evk_reward_normalize(void *state, const float *raw, int64_t n, float sigma_min, float clip,
+                         float *rewards_out, void *stream) {
+    if (!state || !aligned(state, 8) || n < 0 || !(sigma_min > 0.0f) || !(clip >= 0.0f)) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!raw || !rewards_out) return EVK_ERR_INVALID;
+    return cuda_status(launch_reward_normalize(static_cast<double *>(state), raw, n, sigma_min, clip, rewards_out,
+                                               static_cast<cudaStream_t>(stream)));
+}
+
 int evk_last_status(evk_mem *mem, void *stream_v) {
     if (!mem) return EVK_ERR_INVALID;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);

@@ -78,4 +78,11 @@ int64_t q_update_static_max();
 cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
                                    int64_t m, float alpha, int32_t *status, cudaStream_t stream, int *launches);
 
+// ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
+cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);
+cudaError_t launch_reward_refine(const float *best, const float *latency, const uint8_t *feasible, int64_t n,
+                                 float *out, cudaStream_t stream);
+cudaError_t launch_reward_normalize(double *state, const float *raw, int64_t n, float sigma_min, float clip,
+                                    float *out, cudaStream_t stream);
+
 }  // namespace evk

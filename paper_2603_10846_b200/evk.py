@@ -42,7 +42,8 @@ EXPORTS = (
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
-    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_last_status",
+    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_reward_draft",
+    "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
     "evk_launch_count", "evk_strerror",
 )
 
@@ -89,6 +90,11 @@ def _load() -> ctypes.CDLL:
         "evk_q_update_host": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
         "evk_retrieve_plan": (cint, [vp, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]),
         "evk_mem_profile_scoring": (cint, [vp, vp, vp]),
+        "evk_reward_draft": (cint, [vp, i64, vp, vp]),
+        "evk_reward_refine": (cint, [vp, vp, vp, i64, vp, vp]),
+        "evk_reward_norm_state_bytes": (sz, []),
+        "evk_reward_norm_reset": (cint, [vp, vp]),
+        "evk_reward_normalize": (cint, [vp, vp, i64, f32, f32, vp, vp]),
         "evk_last_status": (cint, [vp, vp]),
         "evk_launch_count": (i64, [vp]),
         "evk_strerror": (ctypes.c_char_p, [cint]),
@@ -341,3 +347,39 @@ def evk_mem_profile_scoring(mem: EvkMem, start: Optional[torch.cuda.Event], stop
 
 def evk_last_status(mem: EvkMem, stream=None) -> int:
     return int(_lib.evk_last_status(mem.handle, _stream_ptr(stream)))
+
+
+def evk_reward_draft(feasible: torch.Tensor, stream=None) -> torch.Tensor:
+    """Eq. 5: +1 where feasible else -1.  feasible: uint8 CUDA tensor."""
+    out = torch.empty(feasible.numel(), dtype=torch.float32, device=feasible.device)
+    _check(_lib.evk_reward_draft(_dev(feasible, torch.uint8, "feasible"), feasible.numel(), _dev(out),
+                                 _stream_ptr(stream)), "evk_reward_draft")
+    return out
+
+
+def evk_reward_refine(best_latency: torch.Tensor, latency: torch.Tensor, feasible: torch.Tensor,
+                      stream=None) -> torch.Tensor:
+    """Eq. 6: -1 where infeasible else tanh(log best - log latency)."""
+    n = latency.numel()
+    out = torch.empty(n, dtype=torch.float32, device=latency.device)
+    _check(_lib.evk_reward_refine(_dev(best_latency, torch.float32, "best_latency"),
+                                  _dev(latency, torch.float32, "latency"), _dev(feasible, torch.uint8, "feasible"),
+                                  n, _dev(out), _stream_ptr(stream)), "evk_reward_refine")
+    return out
+
+
+def evk_reward_norm_state(device="cuda", stream=None) -> torch.Tensor:
+    """A fresh (zeroed) running-statistics state for evk_reward_normalize."""
+    state = torch.empty(int(_lib.evk_reward_norm_state_bytes()) // 8, dtype=torch.float64, device=device)
+    _check(_lib.evk_reward_norm_reset(_dev(state), _stream_ptr(stream)), "evk_reward_norm_reset")
+    return state
+
+
+def evk_reward_normalize(state: torch.Tensor, raw: torch.Tensor, sigma_min: float, clip: float = 0.0,
+                         stream=None) -> torch.Tensor:
+    """Running z-score of raw rewards with the statistics seen before each one (Appendix A)."""
+    out = torch.empty(raw.numel(), dtype=torch.float32, device=raw.device)
+    _check(_lib.evk_reward_normalize(_dev(state, torch.float64, "state"), _dev(raw, torch.float32, "raw"),
+                                     raw.numel(), float(sigma_min), float(clip), _dev(out), _stream_ptr(stream)),
+           "evk_reward_normalize")
+    return out
