@@ -66,6 +66,11 @@ def _load():
     lib.evk_oracle_reward_refine.restype = None
     lib.evk_oracle_reward_normalize.argtypes = [p, c_i64, p, c_i64, c_f64, c_f64, p]
     lib.evk_oracle_reward_normalize.restype = None
+    lib.evk_oracle_philox4x32_10.argtypes = [p, p, p]
+    lib.evk_oracle_philox4x32_10.restype = None
+    lib.evk_oracle_explore.argtypes = [p, p, c_i32, p, c_f64, c_i32, c_f32, ctypes.c_uint64, ctypes.c_uint64,
+                                       ctypes.c_uint32, p, p]
+    lib.evk_oracle_explore.restype = c_i32
     _lib = lib
     return lib
 
@@ -203,3 +208,32 @@ def reward_normalize(history, raw, sigma_min: float, clip: float = 0.0) -> np.nd
     out = np.empty(r.shape, dtype=np.float64)
     _load().evk_oracle_reward_normalize(_ptr(h), h.size, _ptr(r), r.size, float(sigma_min), float(clip), _ptr(out))
     return out
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    """One block of Philox4x32-10: counter 4 x uint32, key 2 x uint32 -> 4 x uint32."""
+    c = _c(counter, np.uint32)
+    k = _c(key, np.uint32)
+    out = np.empty(4, dtype=np.uint32)
+    _load().evk_oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def explore(pool_ids, pool_sims, q_stage, w: float, k2: int, epsilon: float, seed: int, step: int,
+            first_query: int = 0):
+    """Epsilon-greedy choice per query over canonical pools; returns (ids, scores, explored)."""
+    pool_ids = _c(pool_ids, np.int32)
+    pool_sims = _c(pool_sims, np.float64)
+    q_stage = _c(q_stage, np.float32)
+    if pool_ids.ndim == 1:
+        pool_ids, pool_sims = pool_ids[None, :], pool_sims[None, :]
+    b, k1 = pool_ids.shape
+    ids = np.empty((b, k2), dtype=np.int32)
+    sc = np.empty((b, k2), dtype=np.float64)
+    explored = np.zeros(b, dtype=np.uint8)
+    lib = _load()
+    for i in range(b):
+        explored[i] = lib.evk_oracle_explore(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage), float(w), k2,
+                                             float(np.float32(epsilon)), int(seed), int(step), first_query + i,
+                                             _ptr(ids[i]), _ptr(sc[i]))
+    return ids, sc, explored

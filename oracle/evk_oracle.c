@@ -217,3 +217,67 @@ void evk_oracle_reward_normalize(const double *history, int64_t n_hist, const fl
         out[t] = r;
     }
 }
+
+/* ---- Exploration: epsilon-greedy choice of the context (Section 3.3) ------------- */
+
+/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+ * SC'11): ten rounds of two 32x32->64 multiplications and key bumps. */
+void evk_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The j-th 32-bit word of the stream of (seed, step, query): block j/4 of the generator
+ * with counter (query, step_lo, step_hi, block) and key (seed_lo, seed_hi). */
+static uint32_t explore_word(uint64_t seed, uint64_t step, uint32_t query, uint32_t j) {
+    const uint32_t ctr[4] = {query, (uint32_t)step, (uint32_t)(step >> 32), j / 4};
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    evk_oracle_philox4x32_10(ctr, key, out);
+    return out[j % 4];
+}
+
+/* Epsilon-greedy over the pool of one query.  Word 0 of the query's stream decides: with
+ * u = (word >> 8) * 2^-24 < epsilon the context is min(k2, n) pool entries drawn uniformly
+ * without replacement (a partial Fisher-Yates shuffle of the pool positions, position i
+ * swapped with i + floor(word_{i+1} * (n - i) / 2^32)), in draw order, each with its mixed
+ * score; otherwise it is the greedy result of evk_oracle_phase2.  The pool must be in its
+ * canonical order (similarity descending, id ascending).  Returns 1 if the query explored. */
+int32_t evk_oracle_explore(const int32_t *pool_ids, const double *pool_sims, int32_t k1,
+                           const float *q_stage, double w, int32_t k2, float epsilon,
+                           uint64_t seed, uint64_t step, uint32_t query,
+                           int32_t *ids_out, double *scores_out) {
+    int32_t n = 0;
+    while (n < k1 && pool_ids[n] >= 0) ++n;
+    const float u = (float)(explore_word(seed, step, query, 0) >> 8) * (1.0f / 16777216.0f);
+    if (!(u < epsilon) || n == 0) {
+        evk_oracle_phase2(pool_ids, pool_sims, k1, q_stage, w, k2, ids_out, scores_out);
+        return 0;
+    }
+    int32_t *perm = (int32_t *)malloc((size_t)n * sizeof(int32_t));
+    for (int32_t i = 0; i < n; ++i) perm[i] = i;
+    const int32_t m = k2 < n ? k2 : n;
+    for (int32_t j = 0; j < k2; ++j) { ids_out[j] = -1; scores_out[j] = -INFINITY; }
+    for (int32_t i = 0; i < m; ++i) {
+        const uint32_t r = explore_word(seed, step, query, (uint32_t)(i + 1));
+        const int32_t pick = i + (int32_t)(((uint64_t)r * (uint64_t)(n - i)) >> 32);
+        const int32_t tmp = perm[i]; perm[i] = perm[pick]; perm[pick] = tmp;
+        const int32_t pos = perm[i];
+        ids_out[i] = pool_ids[pos];
+        scores_out[i] = (1.0 - w) * pool_sims[pos] + w * (double)q_stage[pool_ids[pos]];
+    }
+    free(perm);
+    return 1;
+}
