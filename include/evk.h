@@ -196,6 +196,24 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
                       const float *rewards_host, float alpha,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* evk_retrieve with epsilon-greedy exploration (Section 3.3: the context is drawn from the
+ * pool with an epsilon-greedy policy over the stage's values).  Per query, word 0 of a
+ * Philox4x32-10 stream keyed by (seed; counter = query index, step, block) gives
+ * u = (word >> 8) * 2^-24; if u < epsilon the query explores: its result is min(k2, n) entries
+ * of its pool (n = pool length) drawn uniformly without replacement — a partial Fisher-Yates
+ * shuffle of the pool positions in (sim desc, id asc) order, position i swapped with
+ * i + floor(word_{i+1} * (n - i) / 2^32) — written in draw order with their mixed scores.
+ * Other queries get the greedy result of evk_retrieve.  The draw depends only on (seed,
+ * step, query index): pass a new `step` for every call of an episode.  explored_out [B]
+ * (may be NULL) receives 1 for queries that explored.  epsilon in [0, 1]; epsilon = 0 is
+ * evk_retrieve.  Workspace: evk_retrieve_explore_workspace_bytes(mem, B, k1). */
+size_t evk_retrieve_explore_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1);
+int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage,
+                         int32_t k1, int32_t k2, float w, float epsilon, uint64_t seed, uint64_t step,
+                         int32_t *ids_out, float *scores_out, uint8_t *explored_out,
+                         int32_t *pool_ids_out, float *pool_sims_out,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
 /* Rewards for evk_q_update.  All arrays are device arrays of n elements.
  *
  * evk_reward_draft (Eq. 5): +1 where feasible[i] != 0, else -1.

@@ -383,6 +383,40 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
     return cuda_status(cudaStreamSynchronize(stream));
 }
 
+// ---- exploration -----------------------------------------------------------------
+
+size_t evk_retrieve_explore_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1) {
+    const size_t inner = evk_retrieve_workspace_bytes(mem, B, k1);
+    if (inner == 0) return 0;
+    return inner + 2 * align256((size_t)B * k1 * sizeof(float));
+}
+
+int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage,
+                         int32_t k1, int32_t k2, float w, float epsilon, uint64_t seed, uint64_t step,
+                         int32_t *ids_out, float *scores_out, uint8_t *explored_out,
+                         int32_t *pool_ids_out, float *pool_sims_out,
+                         void *workspace, size_t workspace_bytes, void *stream) {
+    if (!(epsilon >= 0.0f && epsilon <= 1.0f)) return EVK_ERR_INVALID;
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1) return EVK_ERR_INVALID;
+    if (B == 0) return EVK_OK;
+    if (!workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (workspace_bytes < evk_retrieve_explore_workspace_bytes(mem, B, k1)) return EVK_ERR_WORKSPACE;
+    // the pool is needed in its canonical order: use the caller's arrays or scratch of our own
+    char *ws = static_cast<char *>(workspace);
+    const size_t pool_bytes = align256((size_t)B * k1 * sizeof(float));
+    int32_t *pool_ids = pool_ids_out ? pool_ids_out : reinterpret_cast<int32_t *>(ws);
+    float *pool_sims = pool_sims_out ? pool_sims_out : reinterpret_cast<float *>(ws + pool_bytes);
+    int rc = evk_retrieve(mem, queries, q_dtype, B, stage, k1, k2, w, ids_out, scores_out, pool_ids, pool_sims,
+                          ws + 2 * pool_bytes, workspace_bytes - 2 * pool_bytes, stream);
+    if (rc != EVK_OK) return rc;
+    int launches = 0;
+    cudaError_t err = launch_explore(pool_ids, pool_sims, B, k1, k2, mem->q_tables + (size_t)stage * mem->cfg.capacity,
+                                     w, epsilon, seed, step, ids_out, scores_out, explored_out,
+                                     static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
 // ---- rewards -------------------------------------------------------------------
 
 int evk_reward_draft(const uint8_t *feasible, int64_t n, float *rewards_out, void *stream) {

@@ -78,6 +78,12 @@ int64_t q_update_static_max();
 cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
                                    int64_t m, float alpha, int32_t *status, cudaStream_t stream, int *launches);
 
+// ---- epsilon-greedy exploration over the pool -----------------------------------------
+cudaError_t launch_explore(const int32_t *pool_ids, const float *pool_sims, int B, int k1, int k2,
+                           const float *q_stage, float w, float epsilon, uint64_t seed, uint64_t step,
+                           int32_t *ids_out, float *scores_out, uint8_t *explored_out, cudaStream_t stream,
+                           int *launches);
+
 // ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
 cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);
 cudaError_t launch_reward_refine(const float *best, const float *latency, const uint8_t *feasible, int64_t n,

@@ -42,7 +42,8 @@ EXPORTS = (
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
-    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_reward_draft",
+    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
+    "evk_retrieve_explore", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
     "evk_launch_count", "evk_strerror",
 )
@@ -90,6 +91,9 @@ def _load() -> ctypes.CDLL:
         "evk_q_update_host": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
         "evk_retrieve_plan": (cint, [vp, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]),
         "evk_mem_profile_scoring": (cint, [vp, vp, vp]),
+        "evk_retrieve_explore_workspace_bytes": (sz, [vp, i32, i32]),
+        "evk_retrieve_explore": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, f32, ctypes.c_uint64, ctypes.c_uint64,
+                                        vp, vp, vp, vp, vp, vp, sz, vp]),
         "evk_reward_draft": (cint, [vp, i64, vp, vp]),
         "evk_reward_refine": (cint, [vp, vp, vp, i64, vp, vp]),
         "evk_reward_norm_state_bytes": (sz, []),
@@ -383,3 +387,24 @@ def evk_reward_normalize(state: torch.Tensor, raw: torch.Tensor, sigma_min: floa
                                      raw.numel(), float(sigma_min), float(clip), _dev(out), _stream_ptr(stream)),
            "evk_reward_normalize")
     return out
+
+
+def evk_retrieve_explore(mem: EvkMem, queries: torch.Tensor, stage: int, k1: int, k2: int, w: float,
+                         epsilon: float, seed: int, step: int, return_pool: bool = False, stream=None):
+    """evk_retrieve with epsilon-greedy exploration; returns (ids, scores, explored[, pool_ids, pool_sims])."""
+    if queries.dim() != 2 or queries.shape[1] != mem.d:
+        raise ValueError("queries must be [B][d]")
+    B, dev = queries.shape[0], queries.device
+    ids = torch.empty((B, k2), dtype=torch.int32, device=dev)
+    scores = torch.empty((B, k2), dtype=torch.float32, device=dev)
+    explored = torch.empty(B, dtype=torch.uint8, device=dev)
+    pool_ids = torch.empty((B, k1), dtype=torch.int32, device=dev) if return_pool else None
+    pool_sims = torch.empty((B, k1), dtype=torch.float32, device=dev) if return_pool else None
+    ws = mem.workspace("retrieve_explore", int(_lib.evk_retrieve_explore_workspace_bytes(mem.handle, B, k1)))
+    _check(_lib.evk_retrieve_explore(mem.handle, _dev(queries, None, "queries"), _emb_dtype(queries), B, stage,
+                                     k1, k2, float(w), float(epsilon), int(seed), int(step), _dev(ids), _dev(scores),
+                                     _dev(explored), _dev(pool_ids), _dev(pool_sims), _dev(ws), ws.numel(),
+                                     _stream_ptr(stream)), "evk_retrieve_explore")
+    if return_pool:
+        return ids, scores, explored, pool_ids, pool_sims
+    return ids, scores, explored
