@@ -214,6 +214,17 @@ int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t
                          int32_t *pool_ids_out, float *pool_sims_out,
                          void *workspace, size_t workspace_bytes, void *stream);
 
+/* Start-point selection by value (Section 3.4: among the feasible kernels P(x) of a task,
+ * the next start point is chosen with Q_2).  Task t owns the candidate entry ids
+ * cand_ids[offsets[t] .. offsets[t+1]) (device arrays; offsets has n_tasks + 1 elements; ids
+ * distinct within a task, at most 4096 per task).  For every task the k candidates of largest
+ * Q_stage are written to ids_out / q_out [n_tasks][k], ordered (Q descending, id ascending),
+ * padded with id -1 / -inf.  1 <= k <= EVK_MAX_K1.  An id outside [0, size) sets
+ * EVK_ERR_RANGE, a task longer than 4096 EVK_ERR_UNSUPPORTED (status word; that task's row is
+ * all padding). */
+int evk_select_by_value(evk_mem *mem, const int32_t *cand_ids, const int32_t *offsets, int32_t n_tasks, int stage,
+                        int32_t k, int32_t *ids_out, float *q_out, void *stream);
+
 /* Rewards for evk_q_update.  All arrays are device arrays of n elements.
  *
  * evk_reward_draft (Eq. 5): +1 where feasible[i] != 0, else -1.

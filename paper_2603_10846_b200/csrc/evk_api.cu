@@ -417,6 +417,21 @@ int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t
     return cuda_status(err);
 }
 
+// ---- start points ------------------------------------------------------------------
+
+int evk_select_by_value(evk_mem *mem, const int32_t *cand_ids, const int32_t *offsets, int32_t n_tasks, int stage,
+                        int32_t k, int32_t *ids_out, float *q_out, void *stream) {
+    if (!mem || n_tasks < 0 || !stage_ok(mem, stage) || k < 1 || k > EVK_MAX_K1) return EVK_ERR_INVALID;
+    if (n_tasks == 0) return EVK_OK;
+    if (!cand_ids || !offsets || !ids_out || !q_out) return EVK_ERR_INVALID;
+    int launches = 0;
+    cudaError_t err = launch_select_by_value(cand_ids, offsets, n_tasks, mem->size,
+                                             mem->q_tables + (size_t)stage * mem->cfg.capacity, k, ids_out, q_out,
+                                             mem->status, static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
 // ---- rewards -------------------------------------------------------------------
 
 int evk_reward_draft(const uint8_t *feasible, int64_t n, float *rewards_out, void *stream) {

@@ -84,6 +84,11 @@ cudaError_t launch_explore(const int32_t *pool_ids, const float *pool_sims, int 
                            int32_t *ids_out, float *scores_out, uint8_t *explored_out, cudaStream_t stream,
                            int *launches);
 
+// ---- start points by value (Section 3.4) -----------------------------------------------
+cudaError_t launch_select_by_value(const int32_t *cand_ids, const int32_t *offsets, int n_tasks, int64_t size,
+                                   const float *q_stage, int k, int32_t *ids_out, float *q_out, int32_t *status,
+                                   cudaStream_t stream, int *launches);
+
 // ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
 cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);
 cudaError_t launch_reward_refine(const float *best, const float *latency, const uint8_t *feasible, int64_t n,

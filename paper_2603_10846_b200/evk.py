@@ -43,7 +43,7 @@ EXPORTS = (
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
-    "evk_retrieve_explore", "evk_reward_draft",
+    "evk_retrieve_explore", "evk_select_by_value", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
     "evk_launch_count", "evk_strerror",
 )
@@ -94,6 +94,7 @@ def _load() -> ctypes.CDLL:
         "evk_retrieve_explore_workspace_bytes": (sz, [vp, i32, i32]),
         "evk_retrieve_explore": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, f32, ctypes.c_uint64, ctypes.c_uint64,
                                         vp, vp, vp, vp, vp, vp, sz, vp]),
+        "evk_select_by_value": (cint, [vp, vp, vp, i32, cint, i32, vp, vp, vp]),
         "evk_reward_draft": (cint, [vp, i64, vp, vp]),
         "evk_reward_refine": (cint, [vp, vp, vp, i64, vp, vp]),
         "evk_reward_norm_state_bytes": (sz, []),
@@ -408,3 +409,15 @@ def evk_retrieve_explore(mem: EvkMem, queries: torch.Tensor, stage: int, k1: int
     if return_pool:
         return ids, scores, explored, pool_ids, pool_sims
     return ids, scores, explored
+
+
+def evk_select_by_value(mem: EvkMem, cand_ids: torch.Tensor, offsets: torch.Tensor, stage: int, k: int,
+                        stream=None):
+    """Per task, the k candidates of largest Q_stage: (ids [T][k], q [T][k])."""
+    T = offsets.numel() - 1
+    ids = torch.empty((T, k), dtype=torch.int32, device=cand_ids.device)
+    q = torch.empty((T, k), dtype=torch.float32, device=cand_ids.device)
+    _check(_lib.evk_select_by_value(mem.handle, _dev(cand_ids, torch.int32, "cand_ids"),
+                                    _dev(offsets, torch.int32, "offsets"), T, stage, k, _dev(ids), _dev(q),
+                                    _stream_ptr(stream)), "evk_select_by_value")
+    return ids, q
