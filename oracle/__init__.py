@@ -71,6 +71,10 @@ def _load():
     lib.evk_oracle_explore.argtypes = [p, p, c_i32, p, c_f64, c_i32, c_f32, ctypes.c_uint64, ctypes.c_uint64,
                                        ctypes.c_uint32, p, p]
     lib.evk_oracle_explore.restype = c_i32
+    lib.evk_oracle_q_update_decay_f64.argtypes = [p, p, p, p, c_i64]
+    lib.evk_oracle_q_update_decay_f64.restype = None
+    lib.evk_oracle_q_update_decay_f32.argtypes = [p, p, p, p, c_i64]
+    lib.evk_oracle_q_update_decay_f32.restype = None
     _lib = lib
     return lib
 
@@ -237,3 +241,17 @@ def explore(pool_ids, pool_sims, q_stage, w: float, k2: int, epsilon: float, see
                                              float(np.float32(epsilon)), int(seed), int(step), first_query + i,
                                              _ptr(ids[i]), _ptr(sc[i]))
     return ids, sc, explored
+
+
+def q_update_decay(q_stage, visits, ids, rewards, dtype=np.float32):
+    """Eq. 8 with alpha_t = 1/visits (running mean); returns (new table, new visit counts)."""
+    q = np.array(q_stage, dtype=dtype, order="C", copy=True)
+    v = np.array(visits, dtype=np.uint32, order="C", copy=True)
+    ids = _c(ids, np.int32)
+    rewards = _c(rewards, np.float32)
+    assert ids.shape == rewards.shape and ids.ndim == 1 and q.shape == v.shape
+    if ids.size:
+        assert ids.min() >= 0 and ids.max() < q.size
+    fn = _load().evk_oracle_q_update_decay_f32 if dtype == np.float32 else _load().evk_oracle_q_update_decay_f64
+    fn(_ptr(q), _ptr(v), _ptr(ids), _ptr(rewards), ids.size)
+    return q, v

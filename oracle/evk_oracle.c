@@ -281,3 +281,34 @@ int32_t evk_oracle_explore(const int32_t *pool_ids, const double *pool_sims, int
     free(perm);
     return 1;
 }
+
+/* ---- Decreasing step size (Appendix A, Robbins-Monro lemma) ------------------------ */
+
+/* Eq. 8 with alpha_t = 1 / (number of updates the entry has received, this one included):
+ * the stored value becomes the running mean of the entry's rewards.  visits[] counts the
+ * updates per entry and is advanced here.  fp64 truth. */
+void evk_oracle_q_update_decay_f64(double *q_stage, uint32_t *visits, const int32_t *ids,
+                                   const float *rewards, int64_t m) {
+    for (int64_t t = 0; t < m; ++t) {
+        const int32_t i = ids[t];
+        visits[i] += 1;
+        const double alpha = 1.0 / (double)visits[i];
+        q_stage[i] = q_stage[i] + alpha * ((double)rewards[t] - q_stage[i]);
+    }
+}
+
+/* The same in binary32: alpha = 1.0f / (float)visits by IEEE division, then the three
+ * separately rounded operations of evk_oracle_q_update_f32. */
+void evk_oracle_q_update_decay_f32(float *q_stage, uint32_t *visits, const int32_t *ids,
+                                   const float *rewards, int64_t m) {
+    for (int64_t t = 0; t < m; ++t) {
+        const int32_t i = ids[t];
+        visits[i] += 1;
+        volatile float alpha = 1.0f / (float)visits[i];
+        volatile float q = q_stage[i];
+        volatile float diff = rewards[t] - q;
+        volatile float step = alpha * diff;
+        volatile float next = q + step;
+        q_stage[i] = next;
+    }
+}

@@ -405,3 +405,49 @@ def test_update_ema_statistics():
     q = oracle.q_update_f64(np.zeros(n, np.float32), ids, r, a)
     assert abs(q.mean() - mu) < 0.02
     assert abs(q.var() / (a / (2 - a) * sigma ** 2) - 1) < 0.1
+
+
+# --------------------------------------------------------------------------
+# Decreasing step size (Appendix A, Robbins-Monro lemma): alpha_t = 1 / visits
+# --------------------------------------------------------------------------
+
+def test_decay_update_is_the_running_mean():
+    # with alpha_t = 1/t the first update overwrites Q_0 and Q_t is the mean of the rewards so far
+    rng = np.random.default_rng(40)
+    n, m = 30, 2000
+    ids = rng.integers(0, n, m).astype(np.int32)
+    r = (rng.integers(-8, 9, m) / 8).astype(np.float32)
+    q0 = rng.standard_normal(n).astype(np.float32)
+    q64, v = oracle.q_update_decay(q0, np.zeros(n, np.uint32), ids, r, dtype=np.float64)
+    assert v.tolist() == np.bincount(ids, minlength=n).tolist()
+    for i in range(n):
+        hits = r[ids == i]
+        want = Fraction(0)
+        for x in hits:
+            want += Fraction(float(x))
+        if len(hits):
+            assert abs(q64[i] - float(want / len(hits))) < 1e-12
+        else:
+            assert q64[i] == q0[i]
+    # continuing from stored counts equals one long batch; alpha_t satisfies sum = inf, sum of squares < inf
+    qa, va = oracle.q_update_decay(q0, np.zeros(n, np.uint32), ids[:700], r[:700], dtype=np.float32)
+    qb, vb = oracle.q_update_decay(qa, va, ids[700:], r[700:], dtype=np.float32)
+    qc, vc = oracle.q_update_decay(q0, np.zeros(n, np.uint32), ids, r, dtype=np.float32)
+    assert np.array_equal(qb.view(np.uint32), qc.view(np.uint32)) and np.array_equal(vb, vc)
+    assert np.max(np.abs(qc - q64)) < 1e-5
+
+
+def test_decay_update_f32_matches_numpy_scalars_and_converges():
+    rng = np.random.default_rng(41)
+    n, m = 8, 4000
+    ids = rng.integers(0, n, m).astype(np.int32)
+    r = (0.3 + 0.5 * rng.standard_normal(m)).astype(np.float32)
+    q0 = np.zeros(n, np.float32)
+    got, _ = oracle.q_update_decay(q0, np.zeros(n, np.uint32), ids, r)
+    want, cnt = q0.copy(), np.zeros(n, np.int64)
+    for i, rv in zip(ids, r):
+        cnt[i] += 1
+        alpha = np.float32(1.0) / np.float32(cnt[i])
+        want[i] = np.float32(want[i] + np.float32(alpha * np.float32(rv - want[i])))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.max(np.abs(got - 0.3)) < 0.1          # lemma: Q_t -> mu
