@@ -70,7 +70,7 @@ typedef struct evk_config {
 } evk_config;
 
 /* Bytes of device memory a bank of this shape needs (embeddings as bf16 rows
- * [capacity][d], value tables fp32 [n_stages][capacity], a status word).  0 if the
+ * [capacity][d], value tables fp32 and update counts uint32 [n_stages][capacity], a status word).  0 if the
  * config is invalid.  `arena` and `arena_bytes` are ignored. */
 size_t evk_mem_bytes_required(const evk_config *cfg);
 
@@ -173,6 +173,17 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
 enum { EVK_Q_UPDATE_STATIC_MAX = 65536 };
 int evk_q_update_static(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
                         const float *rewards, float alpha, void *stream);
+
+/* The value update with a decreasing step size (Appendix A, Eq. 8 with alpha_t under the
+ * Robbins-Monro conditions): alpha_t = 1 / (number of decay updates the entry has received at
+ * this stage, this one included), so the stored value is the running mean of those rewards and
+ * the first such update replaces the initial value.  Same ordering, arithmetic (alpha_t by
+ * IEEE division in binary32, then subtract / multiply / add), checks and workspace as
+ * evk_q_update.  The per-entry counts live in the arena, start at 0 at insert, are advanced
+ * only by this call, and can be read with evk_visits_read (uint32 [n]). */
+int evk_q_update_decay(evk_mem *mem, const int32_t *ids, int64_t M, int stage, const float *rewards,
+                       void *workspace, size_t workspace_bytes, void *stream);
+int evk_visits_read(evk_mem *mem, int stage, int64_t first, int64_t n, uint32_t *out, void *stream);
 
 /* Copy Q_stage[first .. first+n) to / from a device array. */
 int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream);

@@ -13,6 +13,7 @@ struct evk_mem {
     int64_t size;
     __nv_bfloat16 *bank;  // [capacity][d]
     float *q_tables;      // [n_stages][capacity]
+    uint32_t *visits;     // [n_stages][capacity] updates received (decreasing step size)
     int32_t *status;      // device status word
     int scoring;
     int64_t launches;
@@ -24,7 +25,7 @@ namespace {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct ArenaLayout {
-    size_t bank, q_tables, status, total;
+    size_t bank, q_tables, visits, status, total;
 };
 
 bool config_ok(const evk_config *c) {
@@ -37,7 +38,8 @@ ArenaLayout arena_layout(const evk_config *c) {
     ArenaLayout l;
     l.bank = 0;
     l.q_tables = align256((size_t)c->capacity * c->d * sizeof(__nv_bfloat16));
-    l.status = l.q_tables + align256((size_t)c->n_stages * c->capacity * sizeof(float));
+    l.visits = l.q_tables + align256((size_t)c->n_stages * c->capacity * sizeof(float));
+    l.status = l.visits + align256((size_t)c->n_stages * c->capacity * sizeof(uint32_t));
     l.total = l.status + 256;
     return l;
 }
@@ -110,6 +112,7 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     char *base = static_cast<char *>(cfg->arena);
     m->bank = reinterpret_cast<__nv_bfloat16 *>(base + l.bank);
     m->q_tables = reinterpret_cast<float *>(base + l.q_tables);
+    m->visits = reinterpret_cast<uint32_t *>(base + l.visits);
     m->status = reinterpret_cast<int32_t *>(base + l.status);
     m->scoring = EVK_SCORING_AUTO;
     m->launches = 0;
@@ -147,7 +150,7 @@ int evk_mem_insert(evk_mem *mem, const void *emb, int emb_dtype, int64_t n, int 
     if (!emb || !aligned(emb, 16)) return EVK_ERR_INVALID;
     if (mem->size + n > mem->cfg.capacity) return EVK_ERR_CAPACITY;
     int launches = 0;
-    cudaError_t err = launch_insert(mem->bank, mem->q_tables, mem->status, mem->cfg.capacity, mem->cfg.d,
+    cudaError_t err = launch_insert(mem->bank, mem->q_tables, mem->visits, mem->cfg.capacity, mem->cfg.d,
                                     mem->cfg.n_stages, mem->size, n, emb, emb_dtype, stage, q_init,
                                     mem->cfg.q_default, ids_out, static_cast<cudaStream_t>(stream), &launches);
     mem->launches += launches;
@@ -272,9 +275,34 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
     if (workspace_bytes < q_update_workspace_bytes(M)) return EVK_ERR_WORKSPACE;
     int launches = 0;
     cudaError_t err = launch_q_update(mem->q_tables + (size_t)stage * mem->cfg.capacity, mem->size, ids, rewards,
-                                      M, alpha, mem->status, workspace, static_cast<cudaStream_t>(stream), &launches);
+                                      M, alpha, nullptr, mem->status, workspace, static_cast<cudaStream_t>(stream),
+                                      &launches);
     mem->launches += launches;
     return cuda_status(err);
+}
+
+int evk_q_update_decay(evk_mem *mem, const int32_t *ids, int64_t M, int stage, const float *rewards,
+                       void *workspace, size_t workspace_bytes, void *stream) {
+    if (!mem || M < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (M == 0) return EVK_OK;
+    if (M >= ((int64_t)1 << 31)) return EVK_ERR_UNSUPPORTED;
+    if (!ids || !rewards || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (workspace_bytes < q_update_workspace_bytes(M)) return EVK_ERR_WORKSPACE;
+    int launches = 0;
+    const size_t off = (size_t)stage * mem->cfg.capacity;
+    cudaError_t err = launch_q_update(mem->q_tables + off, mem->size, ids, rewards, M, 1.0f, mem->visits + off,
+                                      mem->status, workspace, static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+int evk_visits_read(evk_mem *mem, int stage, int64_t first, int64_t n, uint32_t *out, void *stream) {
+    if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!out) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemcpyAsync(out, mem->visits + (size_t)stage * mem->cfg.capacity + first,
+                                       (size_t)n * sizeof(uint32_t), cudaMemcpyDeviceToDevice,
+                                       static_cast<cudaStream_t>(stream)));
 }
 
 int evk_q_update_static(evk_mem *mem, const int32_t *ids, int64_t M, int stage,

@@ -9,7 +9,7 @@
 namespace evk {
 
 // ---- insert (Eq. 1) ---------------------------------------------------------
-cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, int32_t *status, int64_t capacity,
+cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits, int64_t capacity,
                           int d, int n_stages, int64_t first, int64_t n, const void *emb, int emb_dtype,
                           int stage, const float *q_init, float q_default, int32_t *ids_out,
                           cudaStream_t stream, int *launches);
@@ -69,8 +69,10 @@ cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_count
 
 // ---- Eq. 4 update -----------------------------------------------------------
 size_t q_update_workspace_bytes(int64_t m);
+// visits == nullptr: constant step size alpha.  Otherwise alpha_t = 1 / visits[id] after counting
+// the update (decreasing step size), and the counts are advanced.
 cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
-                            int64_t m, float alpha, int32_t *status, void *workspace,
+                            int64_t m, float alpha, uint32_t *visits, int32_t *status, void *workspace,
                             cudaStream_t stream, int *launches);
 
 // Eq. 4 update with scratch held in a static device array (no caller workspace).

@@ -33,12 +33,15 @@ insert_rows_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src
 }
 
 __global__ void __launch_bounds__(kThreads)
-insert_values_kernel(float *__restrict__ q_tables, int64_t capacity, int n_stages, int64_t first, int64_t n,
+insert_values_kernel(float *__restrict__ q_tables, uint32_t *__restrict__ visits, int64_t capacity, int n_stages,
+                     int64_t first, int64_t n,
                      int stage, const float *__restrict__ q_init, float q_default, int32_t *__restrict__ ids_out) {
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kThreads) {
         const float v = q_init ? q_init[i] : q_default;
-        for (int s = 0; s < n_stages; ++s)
+        for (int s = 0; s < n_stages; ++s) {
             q_tables[(int64_t)s * capacity + first + i] = (stage < 0 || s == stage) ? v : q_default;
+            visits[(int64_t)s * capacity + first + i] = 0;  // no update seen yet
+        }
         if (ids_out) ids_out[i] = (int32_t)(first + i);
     }
 }
@@ -53,18 +56,17 @@ int grid_for(int64_t work_items) {
 
 }  // namespace
 
-cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, int32_t *status, int64_t capacity,
+cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits, int64_t capacity,
                           int d, int n_stages, int64_t first, int64_t n, const void *emb, int emb_dtype,
                           int stage, const float *q_init, float q_default, int32_t *ids_out,
                           cudaStream_t stream, int *launches) {
-    (void)status;
     if (n <= 0) return cudaSuccess;
     const int64_t n_vec = n * d / 8;
     insert_rows_kernel<<<grid_for(n_vec), kThreads, 0, stream>>>(bank + first * d, emb, emb_dtype == EVK_DTYPE_BF16, n_vec);
     ++*launches;
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    insert_values_kernel<<<grid_for(n), kThreads, 0, stream>>>(q_tables, capacity, n_stages, first, n, stage, q_init, q_default, ids_out);
+    insert_values_kernel<<<grid_for(n), kThreads, 0, stream>>>(q_tables, visits, capacity, n_stages, first, n, stage, q_init, q_default, ids_out);
     ++*launches;
     return cudaGetLastError();
 }

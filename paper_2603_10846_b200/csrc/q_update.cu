@@ -160,7 +160,8 @@ radix_scatter_kernel(const int32_t *__restrict__ keys_in, const float *__restric
 // One thread per run of equal ids (the thread at the run's first element).
 __global__ void __launch_bounds__(kThreads)
 apply_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int64_t m, float alpha,
-             float *__restrict__ q_stage, const int *__restrict__ flags, int32_t *__restrict__ status) {
+             float *__restrict__ q_stage, uint32_t *__restrict__ visits, const int *__restrict__ flags,
+             int32_t *__restrict__ status) {
     const int f = *flags;
     if (f) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && *status == 0)
@@ -182,11 +183,14 @@ apply_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards,
         end = hi;
     }
     float q = q_stage[id];
+    uint32_t seen = visits ? visits[id] : 0;
     for (int64_t j = t; j < end; ++j) {
+        const float a = visits ? __fdiv_rn(1.0f, __uint2float_rn(++seen)) : alpha;
         const float diff = __fsub_rn(rewards[j], q);
-        const float step = __fmul_rn(alpha, diff);
+        const float step = __fmul_rn(a, diff);
         q = __fadd_rn(q, step);
     }
+    if (visits) visits[id] = seen;
     q_stage[id] = q;
 }
 
@@ -198,7 +202,8 @@ constexpr int kSmallMax = 8192;
 
 __global__ void __launch_bounds__(kSmallThreads)
 small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int m, int n_pow2,
-                    int64_t size, float alpha, float *__restrict__ q_stage, int32_t *__restrict__ status) {
+                    int64_t size, float alpha, float *__restrict__ q_stage, uint32_t *__restrict__ visits,
+                    int32_t *__restrict__ status) {
     extern __shared__ __align__(16) unsigned char small_smem[];
     uint64_t *keys = reinterpret_cast<uint64_t *>(small_smem);        // [n_pow2] (id << 32) | position
     float *r = reinterpret_cast<float *>(keys + n_pow2);               // [m]
@@ -249,12 +254,16 @@ small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ r
         const uint32_t id = (uint32_t)(keys[t] >> 32);
         if (t > 0 && (uint32_t)(keys[t - 1] >> 32) == id) continue;  // not the head of its run
         float q = q_stage[id];
+        uint32_t seen = visits ? visits[id] : 0;
         for (int j = t; j < m && (uint32_t)(keys[j] >> 32) == id; ++j) {
+            // decreasing step size: alpha_t = 1 / (updates this entry has received, this one included)
+            const float a = visits ? __fdiv_rn(1.0f, __uint2float_rn(++seen)) : alpha;
             const float diff = __fsub_rn(r[(uint32_t)keys[j]], q);
-            const float step = __fmul_rn(alpha, diff);
+            const float step = __fmul_rn(a, diff);
             q = __fadd_rn(q, step);
         }
         q_stage[id] = q;
+        if (visits) visits[id] = seen;
     }
 }
 
@@ -283,7 +292,7 @@ UpdateLayout layout_for(int64_t m) {
 size_t q_update_workspace_bytes(int64_t m) { return layout_for(m).total; }
 
 cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
-                            int64_t m, float alpha, int32_t *status, void *workspace,
+                            int64_t m, float alpha, uint32_t *visits, int32_t *status, void *workspace,
                             cudaStream_t stream, int *launches) {
     if (m <= 0) return cudaSuccess;
     if (m <= kSmallMax) {
@@ -295,7 +304,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
         if (e != cudaSuccess) return e;
         ++*launches;
         return launch_overlapped(small_update_kernel, dim3(1), dim3(kSmallThreads), smem, stream, ids, rewards, (int)m,
-                                 n_pow2, size, alpha, q_stage, status);
+                                 n_pow2, size, alpha, q_stage, visits, status);
     }
     const UpdateLayout l = layout_for(m);
     char *ws = static_cast<char *>(workspace);
@@ -329,7 +338,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
         k_in = k_out;
         v_in = v_out;
     }
-    apply_kernel<<<(int)((m + kThreads - 1) / kThreads), kThreads, 0, stream>>>(k_in, v_in, m, alpha, q_stage, flags, status);
+    apply_kernel<<<(int)((m + kThreads - 1) / kThreads), kThreads, 0, stream>>>(k_in, v_in, m, alpha, q_stage, visits, flags, status);
     ++*launches;
     return cudaGetLastError();
 }
@@ -378,7 +387,7 @@ cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *
     if (err != cudaSuccess) return err;
     // launch_q_update clears the flag word itself and overwrites every other part of the
     // scratch it reads, so what the previous call left behind does not matter.
-    return launch_q_update(q_stage, size, ids, rewards, m, alpha, status, scratch, stream, launches);
+    return launch_q_update(q_stage, size, ids, rewards, m, alpha, nullptr, status, scratch, stream, launches);
 }
 
 }  // namespace evk

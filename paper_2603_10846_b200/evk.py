@@ -40,7 +40,7 @@ EVK_MAX_K1 = 1024
 EXPORTS = (
     "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
-    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_read", "evk_q_write", "evk_bank_read",
+    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
     "evk_retrieve_explore", "evk_select_by_value", "evk_reward_draft",
@@ -82,6 +82,8 @@ def _load() -> ctypes.CDLL:
         "evk_q_update_workspace_bytes": (sz, [vp, i64]),
         "evk_q_update": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
         "evk_q_update_static": (cint, [vp, vp, i64, cint, vp, f32, vp]),
+        "evk_q_update_decay": (cint, [vp, vp, i64, cint, vp, vp, sz, vp]),
+        "evk_visits_read": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_q_read": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_q_write": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_bank_read": (cint, [vp, i64, i64, vp, vp]),
@@ -421,3 +423,21 @@ def evk_select_by_value(mem: EvkMem, cand_ids: torch.Tensor, offsets: torch.Tens
                                     _dev(offsets, torch.int32, "offsets"), T, stage, k, _dev(ids), _dev(q),
                                     _stream_ptr(stream)), "evk_select_by_value")
     return ids, q
+
+
+def evk_q_update_decay(mem: EvkMem, ids: torch.Tensor, stage: int, rewards: torch.Tensor, stream=None) -> None:
+    """Value update with alpha_t = 1 / visits (running mean of an entry's rewards)."""
+    M = ids.numel()
+    if rewards.numel() != M:
+        raise ValueError("ids and rewards must have the same length")
+    ws = mem.workspace("q_update", evk_q_update_workspace_bytes(mem, M))
+    _check(_lib.evk_q_update_decay(mem.handle, _dev(ids, torch.int32, "ids"), M, stage,
+                                   _dev(rewards, torch.float32, "rewards"), _dev(ws), ws.numel(),
+                                   _stream_ptr(stream)), "evk_q_update_decay")
+
+
+def evk_visits_read(mem: EvkMem, stage: int, first: int = 0, n: Optional[int] = None, stream=None) -> torch.Tensor:
+    n = evk_mem_size(mem) - first if n is None else n
+    out = torch.empty(n, dtype=torch.int32, device=mem.arena.device)
+    _check(_lib.evk_visits_read(mem.handle, stage, first, n, _dev(out), _stream_ptr(stream)), "evk_visits_read")
+    return out
