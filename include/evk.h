@@ -184,6 +184,7 @@ int evk_q_update_static(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
 int evk_q_update_decay(evk_mem *mem, const int32_t *ids, int64_t M, int stage, const float *rewards,
                        void *workspace, size_t workspace_bytes, void *stream);
 int evk_visits_read(evk_mem *mem, int stage, int64_t first, int64_t n, uint32_t *out, void *stream);
+int evk_visits_write(evk_mem *mem, int stage, int64_t first, int64_t n, const uint32_t *values, void *stream);
 
 /* Copy Q_stage[first .. first+n) to / from a device array. */
 int evk_q_read(evk_mem *mem, int stage, int64_t first, int64_t n, float *out, void *stream);

@@ -296,6 +296,15 @@ int evk_q_update_decay(evk_mem *mem, const int32_t *ids, int64_t M, int stage, c
     return cuda_status(err);
 }
 
+int evk_visits_write(evk_mem *mem, int stage, int64_t first, int64_t n, const uint32_t *values, void *stream) {
+    if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!values) return EVK_ERR_INVALID;
+    return cuda_status(cudaMemcpyAsync(mem->visits + (size_t)stage * mem->cfg.capacity + first, values,
+                                       (size_t)n * sizeof(uint32_t), cudaMemcpyDeviceToDevice,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
 int evk_visits_read(evk_mem *mem, int stage, int64_t first, int64_t n, uint32_t *out, void *stream) {
     if (!mem || !stage_ok(mem, stage) || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
     if (n == 0) return EVK_OK;

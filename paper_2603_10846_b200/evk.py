@@ -40,7 +40,7 @@ EVK_MAX_K1 = 1024
 EXPORTS = (
     "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
     "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
-    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_q_read", "evk_q_write", "evk_bank_read",
+    "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_visits_write", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
     "evk_retrieve_explore", "evk_select_by_value", "evk_reward_draft",
@@ -84,6 +84,7 @@ def _load() -> ctypes.CDLL:
         "evk_q_update_static": (cint, [vp, vp, i64, cint, vp, f32, vp]),
         "evk_q_update_decay": (cint, [vp, vp, i64, cint, vp, vp, sz, vp]),
         "evk_visits_read": (cint, [vp, cint, i64, i64, vp, vp]),
+        "evk_visits_write": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_q_read": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_q_write": (cint, [vp, cint, i64, i64, vp, vp]),
         "evk_bank_read": (cint, [vp, i64, i64, vp, vp]),
@@ -441,3 +442,15 @@ def evk_visits_read(mem: EvkMem, stage: int, first: int = 0, n: Optional[int] = 
     out = torch.empty(n, dtype=torch.int32, device=mem.arena.device)
     _check(_lib.evk_visits_read(mem.handle, stage, first, n, _dev(out), _stream_ptr(stream)), "evk_visits_read")
     return out
+
+
+def evk_visits_write(mem: EvkMem, visits, device=None, stream=None) -> None:
+    """Restore per-stage update counts: visits is [n_stages][size] (numpy uint32 or int32 tensor)."""
+    import numpy as _np
+    dev = device or mem.arena.device
+    for s in range(mem.n_stages):
+        row = visits[s]
+        t = row if isinstance(row, torch.Tensor) else torch.from_numpy(_np.ascontiguousarray(row).view(_np.int32))
+        t = t.to(dev).contiguous()
+        _check(_lib.evk_visits_write(mem.handle, s, 0, t.numel(), _dev(t, torch.int32, "visits"),
+                                     _stream_ptr(stream)), "evk_visits_write")
