@@ -30,6 +30,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "retrieval queries/sec at N=1M, d=1024 bf16"
+SCAN_DRAM_BYTES_PER_ENTRY = 543.29e6 / 262224      # d = 1024: 2,071.9 B against 2,048 B algorithmic
 UNIT = "queries/s"
 
 
@@ -319,6 +320,10 @@ def run_evk(args):
         launch_ms = statistics.mean(score_ms) / max(n_score_launches, 1)
         achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
         flops_per_launch = 2.0 * queries_per_launch * size * wl.d
+        # DRAM bytes per launch: read + written bytes per bank entry from one ncu capture of the scan
+        # kernel on a 262,224-row case (profiles/score_mma_clustered_b64.md), scaled by the rows scanned
+        # (the bank is read once, so traffic grows with the rows); unknown for the streaming kernel
+        traffic = SCAN_DRAM_BYTES_PER_ENTRY * size if (kind == evk.EVK_SCORING_TENSOR and wl.d == 1024) else None
         tflops = flops_per_launch / (launch_ms * 1e-3) / 1e12
         # arithmetic intensity of a scan is `queries_per_launch` flop per byte; the ridge of this
         # machine sits near 256, beyond it the tensor cores bound the kernel
@@ -329,7 +334,7 @@ def run_evk(args):
                     "peak": tensor_peak if tensor_bound else peaks["hbm_gbs"],
                     "unit": "TFLOP/s" if tensor_bound else "GB/s",
                     "frac": (tflops / tensor_peak) if tensor_bound else achieved / peaks["hbm_gbs"],
-                    "traffic": None, "peak_source": peaks["source"], "gbs": achieved,
+                    "traffic": traffic, "peak_source": peaks["source"], "gbs": achieved,
                     "kernel": "score_stream" if kind == evk.EVK_SCORING_STREAM else "score_mma",
                     "launches_per_step": n_score_launches, "ms_per_launch": launch_ms,
                     "tflops": flops_per_launch / (launch_ms * 1e-3) / 1e12}
