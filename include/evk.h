@@ -269,6 +269,13 @@ int evk_retrieve_plan(const evk_mem *mem, int32_t B, int32_t k1, int32_t *kind_o
  * setting is used by one call and then cleared; NULLs clear it. */
 int evk_mem_profile_scoring(evk_mem *mem, void *start_event, void *stop_event);
 
+/* Failure-detection test aid.  The next evk_retrieve that runs the tensor kernel starves its
+ * own pipeline: the producer warp issues no loads, so the consumer's bounded wait (shortened to
+ * about a tenth of a second for this call) runs out.  Nothing faults or hangs: every block
+ * raises its abort flag, releases tensor memory and returns, the status word becomes
+ * EVK_ERR_DEVICE_TIMEOUT, that call's outputs are padding, and the handle stays usable. */
+int evk_mem_inject_stall(evk_mem *mem);
+
 /* Synchronise `stream`, return the device status word (EVK_OK or the first
  * device-detected error since the last read) and clear it. */
 int evk_last_status(evk_mem *mem, void *stream);

@@ -16,6 +16,7 @@ struct evk_mem {
     uint32_t *visits;     // [n_stages][capacity] updates received (decreasing step size)
     int32_t *status;      // device status word
     int scoring;
+    int stall_next;       // evk_mem_inject_stall: the next tensor-path retrieve starves its consumer
     int64_t launches;
     cudaEvent_t prof_start, prof_stop;  // armed by evk_mem_profile_scoring for one retrieve
 };
@@ -115,6 +116,7 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     m->visits = reinterpret_cast<uint32_t *>(base + l.visits);
     m->status = reinterpret_cast<int32_t *>(base + l.status);
     m->scoring = EVK_SCORING_AUTO;
+    m->stall_next = 0;
     m->launches = 0;
     m->prof_start = m->prof_stop = nullptr;
     cudaError_t err = cudaMemsetAsync(m->status, 0, 256, 0);
@@ -135,6 +137,12 @@ int evk_mem_destroy(evk_mem *mem) {
 int64_t evk_mem_size(const evk_mem *mem) { return mem ? mem->size : 0; }
 
 int64_t evk_launch_count(const evk_mem *mem) { return mem ? mem->launches : 0; }
+
+int evk_mem_inject_stall(evk_mem *mem) {
+    if (!mem) return EVK_ERR_INVALID;
+    mem->stall_next = 1;
+    return EVK_OK;
+}
 
 int evk_mem_set_scoring(evk_mem *mem, int mode) {
     if (!mem || mode < EVK_SCORING_AUTO || mode > EVK_SCORING_TENSOR) return EVK_ERR_INVALID;
@@ -202,7 +210,9 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     int nparts = 0, part_stride = k1, qt_size = 1;
     if (err == cudaSuccess && mem->size > 0) {
         if (kind == EVK_SCORING_TENSOR) {
-            const MmaPlan plan = mma_plan(mem->size, B, k1);
+            MmaPlan plan = mma_plan(mem->size, B, k1);
+            plan.stall = mem->stall_next;
+            mem->stall_next = 0;
             uint64_t *cand = nullptr;
             int *cand_cnt = nullptr;
             err = launch_score_mma(mem->bank, mem->size, mem->cfg.capacity, mem->cfg.d, q_bf16, B, k1, plan,

@@ -45,6 +45,7 @@ struct MmaPlan {
     int grid;               // thread blocks
     int n_sample;           // 0: no sampling pass
     int64_t sample_stride;  // rows between sampled entries
+    int stall;              // test aid, see evk_mem_inject_stall
 };
 bool mma_supported(int d, int k1);
 MmaPlan mma_plan(int64_t size, int B, int k1);

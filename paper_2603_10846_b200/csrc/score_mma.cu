@@ -88,6 +88,7 @@ struct MmaParams {
     float *dense;       // [B][dense_ld]
     int dense_ld;
     int32_t *status;
+    int stall;          // test aid: the producer of the full scan issues no loads, so a bounded wait runs out
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -113,12 +114,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait; false means the block is aborting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kTimeoutCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -294,6 +295,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long wait_limit = p.stall ? kTimeoutCycles / 16 : kTimeoutCycles;
     pdl_trigger();
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
     const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16, afull = tempty0 + 16;
@@ -326,8 +328,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // ===== TMA producer =====
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
-            bool ok = true;
-            if (p.a_resident && blockIdx.x < n_jobs) {
+            bool ok = !(p.stall && p.mode == 0);
+            if (ok && p.a_resident && blockIdx.x < n_jobs) {
                 mbar_arrive_expect_tx(afull, a_region);
                 for (int kc = 0; kc < k_chunks; ++kc) tma_load_2d(tiles + kc * a_slice, &map_q, afull, kc * kBlockK, 0);
             }
@@ -335,7 +337,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int qt = job / p.splits, split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                     for (int kc = 0; kc < k_chunks; ++kc) {
-                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                         const uint32_t s_dst = ring + stage * stage_bytes;
                         mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
                         if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
@@ -350,15 +352,15 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            if (p.a_resident && blockIdx.x < n_jobs) ok = mbar_wait(afull, 0, abort_flag);
+            if (p.a_resident && blockIdx.x < n_jobs) ok = mbar_wait(afull, 0, abort_flag, wait_limit);
             for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
                 const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
-                    if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * kBlockN;
                     for (int kc = 0; kc < k_chunks; ++kc) {
-                        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, wait_limit)) { ok = false; break; }
                         tc_fence_after();
                         // a resident query tile narrower than 128 rows is read past its end: the
                         // surplus accumulator rows belong to no query and are never looked at
@@ -419,7 +421,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             int cnt = 0;
             uint64_t *my_buf = p.cand + ((size_t)job * kBlockM + m) * kMmaCandCap;
             for (int t = split; t < p.n_tiles && ok; t += p.splits) {
-                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
                 const int64_t row0 = (int64_t)t * kBlockN;
@@ -522,6 +524,10 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
             if (p.mode == 0 && ok) p.cand_cnt[(size_t)job * kBlockM + m] = cnt;
+        }
+        if (!ok && p.mode == 0) {
+            // aborting: whatever this block was to deliver counts as empty, so the merge reads nothing stale
+            for (int job = blockIdx.x; job < n_jobs; job += gridDim.x) p.cand_cnt[(size_t)job * kBlockM + m] = 0;
         }
     }
 
@@ -709,6 +715,7 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     // a strided sample of the bank gives each query a starting threshold
     pl.n_sample = (size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
     pl.sample_stride = pl.n_sample ? size / pl.n_sample : 0;
+    pl.stall = 0;
     return pl;
 }
 
@@ -743,6 +750,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.dense = dense;
     p.dense_ld = kMmaSample;
     p.status = status;
+    p.stall = pl.stall;
     p.tau0 = nullptr;
     p.range = range;
     p.hist = hist;

@@ -39,7 +39,7 @@ EVK_MAX_K1 = 1024
 # Every symbol include/evk.h declares.
 EXPORTS = (
     "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
-    "evk_mem_set_scoring", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
+    "evk_mem_set_scoring", "evk_mem_inject_stall", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_visits_write", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
@@ -76,6 +76,7 @@ def _load() -> ctypes.CDLL:
         "evk_mem_destroy": (cint, [vp]),
         "evk_mem_size": (i64, [vp]),
         "evk_mem_set_scoring": (cint, [vp, cint]),
+        "evk_mem_inject_stall": (cint, [vp]),
         "evk_mem_insert": (cint, [vp, vp, cint, i64, cint, vp, vp, vp]),
         "evk_retrieve_workspace_bytes": (sz, [vp, i32, i32]),
         "evk_retrieve": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]),
@@ -454,3 +455,8 @@ def evk_visits_write(mem: EvkMem, visits, device=None, stream=None) -> None:
         t = t.to(dev).contiguous()
         _check(_lib.evk_visits_write(mem.handle, s, 0, t.numel(), _dev(t, torch.int32, "visits"),
                                      _stream_ptr(stream)), "evk_visits_write")
+
+
+def evk_mem_inject_stall(mem: EvkMem) -> None:
+    """Test aid: the next tensor-path retrieve lets a bounded wait run out (EVK_ERR_DEVICE_TIMEOUT)."""
+    _check(_lib.evk_mem_inject_stall(mem.handle), "evk_mem_inject_stall")

@@ -440,3 +440,21 @@ def test_more_query_tiles_than_sms(evk):
     ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[1], k1, 5, 0.5, out,
                                    sample=[0, 127, 128, 9000, b - 1] + sample_of(b, 40, seed=3))
     assert ep >= 0.9 and ef >= 0.9
+
+
+def test_bounded_wait_runs_out_and_the_handle_survives(evk):
+    # failure detection without a fault: the producer of one scan issues no loads, the consumer's
+    # wait expires, every block backs out, and the status word says so
+    n, d, b = 40000, 256, 20
+    bank = synth.gaussian_unit(n, d, 101, DEV)
+    queries = synth.gaussian_unit(b, d, 102, DEV)
+    q_tab = np.random.default_rng(10).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    good = run_retrieve(evk, mem, queries, 0, 64, 8, 0.5)
+    evk.evk_mem_inject_stall(mem)
+    out = evk.evk_retrieve(mem, queries, 0, 64, 8, 0.5, return_pool=True)
+    assert evk.evk_last_status(mem) == evk.EVK_ERR_DEVICE_TIMEOUT
+    assert torch.all(out[0] == -1) and torch.all(out[2] == -1)
+    again = run_retrieve(evk, mem, queries, 0, 64, 8, 0.5)          # one-shot: the next call is normal
+    for x, y in zip(good, again):
+        assert np.array_equal(x, y)
