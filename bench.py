@@ -272,6 +272,19 @@ def run_evk(args):
     score_ms = [pairs[i][0].elapsed_time(pairs[i][1]) for i in range(0, args.steps, 4)]
     assert evk.evk_last_status(mem) == 0
 
+    # ---- the retrieval alone (scoring + top-k1 + rerank), device-resident, for the roofline of the path ----
+    r_iters = max(10, min(args.steps, 50))
+    r_start, r_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        evk.evk_retrieve(mem, query_sets[i % n_batches], 0, wl.k1, wl.k2, wl.w, out=(ids_out, scores_out))
+    torch.cuda.synchronize()
+    r_start.record(stream)
+    for i in range(r_iters):
+        evk.evk_retrieve(mem, query_sets[i % n_batches], i % 2, wl.k1, wl.k2, wl.w, out=(ids_out, scores_out))
+    r_stop.record(stream)
+    torch.cuda.synchronize()
+    retrieve_ms = r_start.elapsed_time(r_stop) / r_iters
+
     # ---- end to end through the host-buffer entry points ----
     q_host = [query_sets[j % n_batches].cpu().pin_memory() for j in range(4)]
     ids_h = torch.empty((b, wl.k2), dtype=torch.int32).pin_memory()
@@ -351,6 +364,9 @@ def run_evk(args):
             "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": b * wl.d * 2 + n_upd * 8,
                     "d2h_bytes_per_step": b * wl.k2 * 8, "ms_per_step": e2e_ms / e2e_steps},
+            "retrieve_only": {"ms": retrieve_ms, "queries_per_s": b / (retrieve_ms * 1e-3),
+                              "bank_gbs": size * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9,
+                              "frac_of_measured_hbm": size * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
         }
