@@ -237,6 +237,27 @@ int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t
 int evk_select_by_value(evk_mem *mem, const int32_t *cand_ids, const int32_t *offsets, int32_t n_tasks, int stage,
                         int32_t k, int32_t *ids_out, float *q_out, void *stream);
 
+/* A bank split by rows over several GPUs (one process and one evk_mem per GPU).  Shard g
+ * stores the entries with global ids [id_offset_g, id_offset_g + size_g) and their values.
+ *
+ * evk_retrieve_local: phase 1 on this shard for all B queries, each candidate tagged with its
+ *   global id (local id + id_offset) and its Q_stage: gids_out / sims_out / q_out [B][k1],
+ *   ordered (sim desc, id asc), padded with gid -1, sim -inf, q 0.
+ * evk_merge_shards: gids / sims / qs are the gathered outputs of all shards, [n_shards][B][k1],
+ *   shards in ascending id-range order (the caller gathers them, e.g. with an all-gather; the
+ *   arrays are in this GPU's own memory).  Per query: the k1 best of the n_shards * k1
+ *   candidates (sim desc, global id asc) — the pool one unsplit bank would give — then phase 2
+ *   with the values that came along: ids_out (global ids) / scores_out [B][k2], and optionally
+ *   the merged pool [B][k1].  Needs no handle and no workspace.
+ * Updates: each shard applies, in array order, the (id, reward) pairs whose id it owns. */
+size_t evk_retrieve_local_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1);
+int evk_retrieve_local(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage, int32_t k1,
+                       int32_t id_offset, int32_t *gids_out, float *sims_out, float *q_out,
+                       void *workspace, size_t workspace_bytes, void *stream);
+int evk_merge_shards(const int32_t *gids, const float *sims, const float *qs, int32_t n_shards, int32_t B,
+                     int32_t k1, int32_t k2, float w, int32_t *ids_out, float *scores_out,
+                     int32_t *pool_gids_out, float *pool_sims_out, void *stream);
+
 /* Rewards for evk_q_update.  All arrays are device arrays of n elements.
  *
  * evk_reward_draft (Eq. 5): +1 where feasible[i] != 0, else -1.

@@ -479,6 +479,52 @@ int evk_select_by_value(evk_mem *mem, const int32_t *cand_ids, const int32_t *of
     return cuda_status(err);
 }
 
+// ---- row-sharded banks -------------------------------------------------------------
+
+size_t evk_retrieve_local_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1) {
+    const size_t inner = evk_retrieve_workspace_bytes(mem, B, k1);
+    if (inner == 0) return 0;
+    return inner + align256((size_t)B * k1 * sizeof(int32_t)) + 2 * align256((size_t)B * sizeof(float));
+}
+
+int evk_retrieve_local(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int stage, int32_t k1,
+                       int32_t id_offset, int32_t *gids_out, float *sims_out, float *q_out,
+                       void *workspace, size_t workspace_bytes, void *stream) {
+    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || id_offset < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (B == 0) return EVK_OK;
+    if (!gids_out || !sims_out || !q_out || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (workspace_bytes < evk_retrieve_local_workspace_bytes(mem, B, k1)) return EVK_ERR_WORKSPACE;
+    char *ws = static_cast<char *>(workspace);
+    int32_t *pool_ids = reinterpret_cast<int32_t *>(ws);
+    size_t off = align256((size_t)B * k1 * sizeof(int32_t));
+    int32_t *top_ids = reinterpret_cast<int32_t *>(ws + off);
+    off += align256((size_t)B * sizeof(float));
+    float *top_scores = reinterpret_cast<float *>(ws + off);
+    off += align256((size_t)B * sizeof(float));
+    // phase 1 on this shard's rows (the k2 = 1 result is not used)
+    int rc = evk_retrieve(mem, queries, q_dtype, B, stage, k1, 1, 0.0f, top_ids, top_scores, pool_ids, sims_out,
+                          ws + off, workspace_bytes - off, stream);
+    if (rc != EVK_OK) return rc;
+    int launches = 0;
+    cudaError_t err = launch_tag_pool(pool_ids, (int64_t)B * k1, id_offset,
+                                      mem->q_tables + (size_t)stage * mem->cfg.capacity, gids_out, q_out,
+                                      static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+int evk_merge_shards(const int32_t *gids, const float *sims, const float *qs, int32_t n_shards, int32_t B,
+                     int32_t k1, int32_t k2, float w, int32_t *ids_out, float *scores_out,
+                     int32_t *pool_gids_out, float *pool_sims_out, void *stream) {
+    if (n_shards < 1 || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return EVK_ERR_INVALID;
+    if (!(w >= 0.0f && w <= 1.0f)) return EVK_ERR_INVALID;
+    if ((int64_t)n_shards * k1 >= ((int64_t)1 << 31)) return EVK_ERR_UNSUPPORTED;
+    if (B == 0) return EVK_OK;
+    if (!gids || !sims || !qs || !ids_out || !scores_out) return EVK_ERR_INVALID;
+    return cuda_status(launch_merge_shards(gids, sims, qs, n_shards, B, k1, k2, w, ids_out, scores_out,
+                                           pool_gids_out, pool_sims_out, static_cast<cudaStream_t>(stream)));
+}
+
 // ---- rewards -------------------------------------------------------------------
 
 int evk_reward_draft(const uint8_t *feasible, int64_t n, float *rewards_out, void *stream) {

@@ -92,6 +92,13 @@ cudaError_t launch_select_by_value(const int32_t *cand_ids, const int32_t *offse
                                    const float *q_stage, int k, int32_t *ids_out, float *q_out, int32_t *status,
                                    cudaStream_t stream, int *launches);
 
+// ---- a bank split by rows over several GPUs ---------------------------------------------
+cudaError_t launch_tag_pool(const int32_t *pool_ids, int64_t n, int32_t id_offset, const float *q_stage,
+                            int32_t *gids_out, float *q_out, cudaStream_t stream, int *launches);
+cudaError_t launch_merge_shards(const int32_t *gids, const float *sims, const float *qs, int n_shards, int B, int k1,
+                                int k2, float w, int32_t *ids_out, float *scores_out, int32_t *pool_gids_out,
+                                float *pool_sims_out, cudaStream_t stream);
+
 // ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
 cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);
 cudaError_t launch_reward_refine(const float *best, const float *latency, const uint8_t *feasible, int64_t n,

@@ -16,13 +16,18 @@ __device__ __forceinline__ bool rerank_before(uint64_t ka, int32_t ia, uint64_t 
     return ka > kb || (ka == kb && (uint32_t)ia < (uint32_t)ib);
 }
 
-// Block-wide: the pool of one query is n keys in shared memory, in any order.
-// Gathers Q_stage, scores, sorts, writes the first k2 results (padding: id -1, score -inf).
+// One pool entry as the rerank sees it.
+struct PoolEntry {
+    int32_t id;
+    float sim, q;
+};
+
+// Block-wide: scores the n entries that fetch(i) returns (any order), sorts them by (score
+// desc, sim desc, id asc) and writes the first k2 (padding: id -1, score -inf).
 // skey / sid: shared scratch of next_pow2(n) entries each.
-template <int NT>
-__device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const float *__restrict__ q_stage, float w,
-                             uint64_t *skey, int32_t *sid, int32_t *__restrict__ ids_out,
-                             float *__restrict__ scores_out) {
+template <int NT, class Fetch>
+__device__ void rerank_block_with(Fetch fetch, int n, int k2, float w, uint64_t *skey, int32_t *sid,
+                                  int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
     const int tid = threadIdx.x;
     const int np2 = next_pow2(n > 1 ? n : 1);
     const float one_minus_w = 1.0f - w;
@@ -30,11 +35,11 @@ __device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const flo
         uint64_t key = 0;
         int32_t id = -1;  // padding compares as the largest unsigned id and a zero key: last
         if (i < n) {
-            id = key_id(pool_keys[i]);
-            const float sim = key_sim(pool_keys[i]);
-            float score = fmaf(w, q_stage[id], one_minus_w * sim);
+            const PoolEntry e = fetch(i);
+            id = e.id;
+            float score = fmaf(w, e.q, one_minus_w * e.sim);
             score += 0.0f;
-            key = ((uint64_t)ordered_bits(score) << 32) | ordered_bits(sim + 0.0f);
+            key = ((uint64_t)ordered_bits(score) << 32) | ordered_bits(e.sim + 0.0f);
         }
         skey[i] = key;
         sid[i] = id;
@@ -66,6 +71,22 @@ __device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const flo
         ids_out[i] = id;
         scores_out[i] = score;
     }
+}
+
+// The pool as n ranking keys (similarity, id) in shared memory, values looked up in q_stage.
+template <int NT>
+__device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const float *__restrict__ q_stage, float w,
+                             uint64_t *skey, int32_t *sid, int32_t *__restrict__ ids_out,
+                             float *__restrict__ scores_out) {
+    rerank_block_with<NT>(
+        [=](int i) {
+            PoolEntry e;
+            e.id = key_id(pool_keys[i]);
+            e.sim = key_sim(pool_keys[i]);
+            e.q = q_stage[e.id];
+            return e;
+        },
+        n, k2, w, skey, sid, ids_out, scores_out);
 }
 
 }  // namespace evk

@@ -43,7 +43,8 @@ EXPORTS = (
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_visits_write", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
-    "evk_retrieve_explore", "evk_select_by_value", "evk_reward_draft",
+    "evk_retrieve_explore", "evk_select_by_value", "evk_retrieve_local_workspace_bytes", "evk_retrieve_local",
+    "evk_merge_shards", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
     "evk_launch_count", "evk_strerror",
 )
@@ -99,6 +100,9 @@ def _load() -> ctypes.CDLL:
         "evk_retrieve_explore": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, f32, ctypes.c_uint64, ctypes.c_uint64,
                                         vp, vp, vp, vp, vp, vp, sz, vp]),
         "evk_select_by_value": (cint, [vp, vp, vp, i32, cint, i32, vp, vp, vp]),
+        "evk_retrieve_local_workspace_bytes": (sz, [vp, i32, i32]),
+        "evk_retrieve_local": (cint, [vp, vp, cint, i32, cint, i32, i32, vp, vp, vp, vp, sz, vp]),
+        "evk_merge_shards": (cint, [vp, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]),
         "evk_reward_draft": (cint, [vp, i64, vp, vp]),
         "evk_reward_refine": (cint, [vp, vp, vp, i64, vp, vp]),
         "evk_reward_norm_state_bytes": (sz, []),
@@ -460,3 +464,33 @@ def evk_visits_write(mem: EvkMem, visits, device=None, stream=None) -> None:
 def evk_mem_inject_stall(mem: EvkMem) -> None:
     """Test aid: the next tensor-path retrieve lets a bounded wait run out (EVK_ERR_DEVICE_TIMEOUT)."""
     _check(_lib.evk_mem_inject_stall(mem.handle), "evk_mem_inject_stall")
+
+
+def evk_retrieve_local(mem: EvkMem, queries: torch.Tensor, stage: int, k1: int, id_offset: int, stream=None):
+    """Phase 1 on one row shard: (global ids, sims, Q_stage) per candidate, each [B][k1]."""
+    B, dev = queries.shape[0], queries.device
+    gids = torch.empty((B, k1), dtype=torch.int32, device=dev)
+    sims = torch.empty((B, k1), dtype=torch.float32, device=dev)
+    qs = torch.empty((B, k1), dtype=torch.float32, device=dev)
+    ws = mem.workspace("retrieve_local", int(_lib.evk_retrieve_local_workspace_bytes(mem.handle, B, k1)))
+    _check(_lib.evk_retrieve_local(mem.handle, _dev(queries, None, "queries"), _emb_dtype(queries), B, stage, k1,
+                                   int(id_offset), _dev(gids), _dev(sims), _dev(qs), _dev(ws), ws.numel(),
+                                   _stream_ptr(stream)), "evk_retrieve_local")
+    return gids, sims, qs
+
+
+def evk_merge_shards(gids: torch.Tensor, sims: torch.Tensor, qs: torch.Tensor, k2: int, w: float,
+                     return_pool: bool = False, stream=None):
+    """Merge gathered shard pools [G][B][k1] (ascending id ranges) and run phase 2."""
+    G, B, k1 = gids.shape
+    dev = gids.device
+    ids = torch.empty((B, k2), dtype=torch.int32, device=dev)
+    scores = torch.empty((B, k2), dtype=torch.float32, device=dev)
+    pool_g = torch.empty((B, k1), dtype=torch.int32, device=dev) if return_pool else None
+    pool_s = torch.empty((B, k1), dtype=torch.float32, device=dev) if return_pool else None
+    _check(_lib.evk_merge_shards(_dev(gids, torch.int32, "gids"), _dev(sims, torch.float32, "sims"),
+                                 _dev(qs, torch.float32, "qs"), G, B, k1, k2, float(w), _dev(ids), _dev(scores),
+                                 _dev(pool_g), _dev(pool_s), _stream_ptr(stream)), "evk_merge_shards")
+    if return_pool:
+        return ids, scores, pool_g, pool_s
+    return ids, scores

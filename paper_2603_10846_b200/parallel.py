@@ -53,3 +53,35 @@ def gather_update_batches(ids: torch.Tensor, rewards: torch.Tensor,
     dist.all_gather(r_l, pad_r, group=group)
     return (torch.cat([t[:c] for t, c in zip(ids_l, counts)]),
             torch.cat([t[:c] for t, c in zip(r_l, counts)]))
+
+
+# ---- banks too large for one GPU: split by rows -----------------------------------------
+
+def row_shard(n_entries: int, rank: int, world: int) -> Tuple[int, int]:
+    """Contiguous [begin, end) id range of one rank; ranges ascend with the rank."""
+    return shard_queries(n_entries, rank, world)
+
+
+def own_updates(ids: torch.Tensor, rewards: torch.Tensor, begin: int, end: int) -> Tuple[torch.Tensor, torch.Tensor]:
+    """The (id, reward) pairs a shard owns, in array order, with ids made local.  Every rank sees
+    the whole batch; an entry's updates all land on its owner in their original order, so the
+    stored bits equal those of one unsplit table."""
+    mine = (ids >= begin) & (ids < end)
+    return (ids[mine] - begin).to(ids.dtype).contiguous(), rewards[mine].contiguous()
+
+
+def retrieve_row_sharded(evk, mem, queries: torch.Tensor, stage: int, k1: int, k2: int, w: float,
+                         id_offset: int, group: Optional[dist.ProcessGroup] = None):
+    """Retrieval over a row-sharded bank: local phase 1, one all-gather of the tagged pools
+    (B * k1 * 12 bytes per rank), merge + phase 2 on every rank.  Returns global ids and scores."""
+    gids, sims, qs = evk.evk_retrieve_local(mem, queries, stage, k1, id_offset)
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world == 1:
+        return evk.evk_merge_shards(gids[None], sims[None], qs[None], k2, w)
+    all_g = torch.empty((world,) + tuple(gids.shape), dtype=gids.dtype, device=gids.device)
+    all_s = torch.empty((world,) + tuple(sims.shape), dtype=sims.dtype, device=sims.device)
+    all_q = torch.empty((world,) + tuple(qs.shape), dtype=qs.dtype, device=qs.device)
+    dist.all_gather_into_tensor(all_g, gids, group=group)
+    dist.all_gather_into_tensor(all_s, sims, group=group)
+    dist.all_gather_into_tensor(all_q, qs, group=group)
+    return evk.evk_merge_shards(all_g, all_s, all_q, k2, w)

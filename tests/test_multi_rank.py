@@ -61,3 +61,23 @@ def test_query_shards_cover_the_batch():
         assert spans[0][0] == 0 and spans[-1][1] == n
         assert all(a[1] == b[0] for a, b in zip(spans[:-1], spans[1:]))
         assert max(e - b for b, e in spans) - min(e - b for b, e in spans) <= 1
+
+
+def test_row_shards_partition_updates_in_order():
+    # owner-applied updates (ids made local, order kept) give the bits of one unsplit table
+    import oracle
+    n, world, m = 1000, 3, 5000
+    rng = np.random.default_rng(3)
+    ids = np.where(rng.random(m) < 0.3, 400, rng.integers(0, n, m)).astype(np.int32)
+    r = rng.standard_normal(m).astype(np.float32)
+    q0 = rng.random(n).astype(np.float32)
+    want = oracle.q_update_f32(q0, ids, r, 0.2)
+    got = []
+    for rank in range(world):
+        a, e = parallel.row_shard(n, rank, world)
+        li, lr = parallel.own_updates(torch.from_numpy(ids), torch.from_numpy(r), a, e)
+        assert li.numel() == int(((ids >= a) & (ids < e)).sum())
+        got.append(oracle.q_update_f32(q0[a:e], li.numpy(), lr.numpy(), 0.2))
+    assert np.array_equal(np.concatenate(got).view(np.uint32), want.view(np.uint32))
+    spans = [parallel.row_shard(n, rk, world) for rk in range(world)]
+    assert spans[0][0] == 0 and spans[-1][1] == n and all(x[1] == y[0] for x, y in zip(spans[:-1], spans[1:]))
