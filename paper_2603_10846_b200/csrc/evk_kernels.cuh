@@ -43,6 +43,7 @@ struct MmaPlan {
     int n_tiles;            // bank tiles of 256 rows
     int splits;             // bank splits per query tile (= candidate lists per query)
     int grid;               // thread blocks
+    int pair;               // 1: clusters of two blocks share 256-query tiles (cta_group::2)
     int n_sample;           // 0: no sampling pass
     int64_t sample_stride;  // rows between sampled entries
     int stall;              // test aid, see evk_mem_inject_stall

@@ -158,6 +158,60 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ---- two SMs on one tile (cta_group::2) ----------------------------------------------------
+// A cluster of two blocks shares one 256-query x 256-row tile: each block holds its own 128
+// queries (A) and HALF of the bank slice (B), the leader block issues one M=256 instruction
+// that reads both halves, and each block's tensor memory receives the accumulator rows of its
+// own queries.  Per block and slice 16 KB of B travel instead of 32 KB.
+constexpr uint32_t kInstrDescPair = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
+                                    ((uint32_t)(256 >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory offset in block `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this block's shared memory whose bytes are counted on a barrier of the pair's leader
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kInstrDescPair), "r"(accumulate)
+        : "memory");
+}
+// Arrive on the barrier at this offset in BOTH blocks of the pair once the MMAs issued so far finished.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle,
 // 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -272,6 +326,7 @@ __device__ __noinline__ uint64_t warp_select_topk(uint64_t *buf, int n, int k) {
 
 // ---- the kernel ---------------------------------------------------------------
 
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
                  const MmaParams p) {
@@ -280,12 +335,18 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     unsigned char *tiles_ptr = smem_raw + (tiles - raw);
-    const int n_jobs = p.n_qt * p.splits;
+    // kPair: blocks come in clusters of two; `rank` is the block's place in its pair, a "worker" is
+    // a pair.  Otherwise every block is a worker of its own.
+    const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+    const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int n_jobs = (kPair ? (p.n_qt + 1) / 2 : p.n_qt) * p.splits;
     const int k_chunks = p.d / kBlockK;
     // [resident query tile: k_chunks slices of a_rows x 128 B] [ring of n_stages stages] [barriers]
     const uint32_t a_slice = (uint32_t)p.a_rows * 128u;
     const uint32_t a_region = p.a_resident ? (uint32_t)k_chunks * a_slice : 0u;
-    const uint32_t stage_bytes = p.a_resident ? kBBytes : (kABytes + kBBytes);
+    const uint32_t b_bytes = kPair ? kBBytes / 2 : kBBytes;   // this block's share of a bank slice
+    const uint32_t stage_bytes = p.a_resident ? b_bytes : (kABytes + b_bytes);
     const uint32_t b_off = p.a_resident ? 0u : kABytes;   // the bank slice inside a stage
     const uint32_t ring = tiles + a_region;
     const int kStages = p.n_stages;
@@ -308,7 +369,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull0 + 8 * b, 1);
-            mbar_init(tempty0 + 8 * b, 4);
+            mbar_init(tempty0 + 8 * b, kPair ? 8 : 4);  // one arrival per epilogue warp of every block on the tile
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -316,11 +377,17 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     if (warp == 0) {
         __syncwarp();
-        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-        tmem_relinquish();
+        if (kPair) {
+            tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (kPair) cluster_sync_all();  // the partner's barriers exist before anything is signalled across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -329,19 +396,29 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = !(p.stall && p.mode == 0);
-            if (ok && p.a_resident && blockIdx.x < n_jobs) {
+            if (ok && p.a_resident && worker < n_jobs) {
                 mbar_arrive_expect_tx(afull, a_region);
                 for (int kc = 0; kc < k_chunks; ++kc) tma_load_2d(tiles + kc * a_slice, &map_q, afull, kc * kBlockK, 0);
             }
-            for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
-                const int qt = job / p.splits, split = job % p.splits;
+            for (int job = worker; job < n_jobs && ok; job += n_workers) {
+                const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
+                const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                     for (int kc = 0; kc < k_chunks; ++kc) {
                         if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                         const uint32_t s_dst = ring + stage * stage_bytes;
-                        mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
-                        if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
-                        tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
+                        if (kPair) {
+                            // both blocks' bytes are counted on the leader's barrier, which the MMA waits on
+                            const uint32_t leader_full = mapa_u32(full0 + 8 * stage, 0);
+                            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * stage, 2 * stage_bytes);
+                            tma_load_2d_pair(s_dst, &map_q, leader_full, kc * kBlockK, qt * kBlockM);
+                            tma_load_2d_pair(s_dst + b_off, &map_bank, leader_full, kc * kBlockK,
+                                             t * kBlockN + (int)rank * (kBlockN / 2));
+                        } else {
+                            mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
+                            if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
+                            tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
+                        }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                 }
@@ -349,11 +426,11 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else if (warp == 1) {
         // ===== MMA issuer =====
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {  // in a pair only the leader issues
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            if (p.a_resident && blockIdx.x < n_jobs) ok = mbar_wait(afull, 0, abort_flag, wait_limit);
-            for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+            if (p.a_resident && worker < n_jobs) ok = mbar_wait(afull, 0, abort_flag, wait_limit);
+            for (int job = worker; job < n_jobs && ok; job += n_workers) {
                 const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                     if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
@@ -370,14 +447,18 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
                         for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                            umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
-                                      (kc > 0 || k > 0) ? 1u : 0u);
+                            if (kPair)
+                                umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                               (kc > 0 || k > 0) ? 1u : 0u);
+                            else
+                                umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                          (kc > 0 || k > 0) ? 1u : 0u);
                         }
-                        umma_commit(empty0 + 8 * stage);
+                        if (kPair) umma_commit_pair(empty0 + 8 * stage); else umma_commit(empty0 + 8 * stage);
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                     if (!ok) break;
-                    umma_commit(tfull0 + 8 * acc);
+                    if (kPair) umma_commit_pair(tfull0 + 8 * acc); else umma_commit(tfull0 + 8 * acc);
                     if (++acc == 2) { acc = 0; acc_phase ^= 1; }
                 }
             }
@@ -391,8 +472,10 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int m = quarter * 32 + lane;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
-            const int qt = job / p.splits, split = job % p.splits;
+        for (int job = worker; job < n_jobs && ok; job += n_workers) {
+            const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
+            const int split = job % p.splits;
+            const int list_job = qt * p.splits + split;   // candidate lists are per (query tile, split)
             const int q = qt * kBlockM + m;
             const bool q_valid = q < p.B;
             // Two filters, both lower bounds of the query's final k1-th key: the key threshold of this
@@ -419,7 +502,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tau_sim = key_sim_floor;
             }
             int cnt = 0;
-            uint64_t *my_buf = p.cand + ((size_t)job * kBlockM + m) * kMmaCandCap;
+            uint64_t *my_buf = p.cand + ((size_t)list_job * kBlockM + m) * kMmaCandCap;
             for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                 if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
                 tc_fence_after();
@@ -520,14 +603,19 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                if (lane == 0) {
+                    if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * acc, 0)); else mbar_arrive(tempty0 + 8 * acc);
+                }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
-            if (p.mode == 0 && ok) p.cand_cnt[(size_t)job * kBlockM + m] = cnt;
+            if (p.mode == 0 && ok && qt < p.n_qt) p.cand_cnt[(size_t)list_job * kBlockM + m] = cnt;
         }
         if (!ok && p.mode == 0) {
             // aborting: whatever this block was to deliver counts as empty, so the merge reads nothing stale
-            for (int job = blockIdx.x; job < n_jobs; job += gridDim.x) p.cand_cnt[(size_t)job * kBlockM + m] = 0;
+            for (int job = worker; job < n_jobs; job += n_workers) {
+                const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
+                if (qt < p.n_qt) p.cand_cnt[((size_t)qt * p.splits + job % p.splits) * kBlockM + m] = 0;
+            }
         }
     }
 
@@ -540,9 +628,10 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)EVK_ERR_DEVICE_TIMEOUT);
         __syncthreads();
     }
+    if (kPair) cluster_sync_all();  // neither block frees tensor memory or leaves while the other may touch it
     if (warp == 0) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -638,22 +727,38 @@ SmemPlan smem_plan(int B, int d) {
 }
 
 // overlap = true: programmatic dependent launch behind the kernel enqueued just before.
+// pair = true: clusters of two blocks (grid must be even), the cta_group::2 variant.
 cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
-                          size_t smem_bytes, bool overlap, cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+                          size_t smem_bytes, bool overlap, bool pair, cudaStream_t stream) {
+    auto kern = pair ? score_mma_kernel<true> : score_mma_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (overlap) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    if (pair) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 2;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, score_mma_kernel, mq, mb, p);
+    cfg.numAttrs = n_attr;
+    return cudaLaunchKernelEx(&cfg, kern, mq, mb, p);
 }
+
+// Two SMs share a tile when there are at least two query tiles to pair up.
+bool use_pairs(int n_qt) { return n_qt >= 2; }
 
 // Bank splits per query tile.  Jobs (query tile, split) are dealt round-robin to the
 // blocks, one block per SM; the split count is the smallest one from 148 / n_qt upwards whose
@@ -661,14 +766,17 @@ cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const Mm
 // tiles side by side on the same bank tiles (they share them through L2).
 int splits_for(int n_qt, int n_tiles) {
     if (n_qt <= 0) n_qt = 1;
-    int base = kNumSM / n_qt;
+    // workers: single blocks, or pairs of blocks that take two query tiles at a time
+    const int n_work = use_pairs(n_qt) ? kNumSM / 2 : kNumSM;
+    const int n_units = use_pairs(n_qt) ? (n_qt + 1) / 2 : n_qt;
+    int base = n_work / n_units;
     if (base < 1) base = 1;
     int splits = base;
-    if (n_qt < kNumSM) {
-        for (int s = base; s <= 4 * base && s <= kNumSM; ++s) {
-            const int jobs = n_qt * s;
-            const int rounds = (jobs + kNumSM - 1) / kNumSM;
-            if (jobs * 100 >= 97 * rounds * kNumSM) {
+    if (n_units < n_work) {
+        for (int s = base; s <= 4 * base && s <= n_work; ++s) {
+            const int jobs = n_units * s;
+            const int rounds = (jobs + n_work - 1) / n_work;
+            if (jobs * 100 >= 97 * rounds * n_work) {
                 splits = s;
                 break;
             }
@@ -709,8 +817,14 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     pl.n_qt = (B + kBlockM - 1) / kBlockM;
     pl.n_tiles = (int)((size + kBlockN - 1) / kBlockN);
     pl.splits = splits_for(pl.n_qt, pl.n_tiles);
-    const int jobs = pl.n_qt * pl.splits;
-    pl.grid = jobs < kNumSM ? jobs : kNumSM;
+    pl.pair = use_pairs(pl.n_qt) ? 1 : 0;
+    if (pl.pair) {
+        const int jobs = ((pl.n_qt + 1) / 2) * pl.splits;
+        pl.grid = 2 * (jobs < kNumSM / 2 ? jobs : kNumSM / 2);
+    } else {
+        const int jobs = pl.n_qt * pl.splits;
+        pl.grid = jobs < kNumSM ? jobs : kNumSM;
+    }
     if (pl.grid < 1) pl.grid = 1;
     // a strided sample of the bank gives each query a starting threshold
     pl.n_sample = (size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
@@ -765,9 +879,13 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.size = pl.n_sample;
         p.mode = 1;
         p.n_tiles = pl.n_sample / kBlockN;
-        p.splits = splits_for(p.n_qt, p.n_tiles);
+        // the sample pass is small: single blocks, as many splits as fit next to the query tiles
+        int s_splits = kNumSM / p.n_qt;
+        if (s_splits < 1) s_splits = 1;
+        if (s_splits > p.n_tiles) s_splits = p.n_tiles;
+        p.splits = s_splits;
         const int jobs = p.n_qt * p.splits;
-        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, false, stream);
+        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, false, false, stream);
         if (err != cudaSuccess) return err;
         ++*launches;
         {
@@ -788,7 +906,15 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.tau0 = tau0;
     }
 
-    if (!make_map(&map_bank, bank, d, capacity, d, kBlockN)) return cudaErrorInvalidValue;
+    // in a pair every block loads its half of a bank slice (128 rows) and its own query slice
+    if (!make_map(&map_bank, bank, d, capacity, d, pl.pair ? kBlockN / 2 : kBlockN)) return cudaErrorInvalidValue;
+    size_t smem_bytes = sp.bytes;
+    if (pl.pair) {
+        p.a_resident = 0;
+        p.a_rows = kBlockM;
+        p.n_stages = kMaxStages;
+        smem_bytes = kSmemFixed + (size_t)kMaxStages * (kABytes + kBBytes / 2);
+    }
     p.size = size;
     p.mode = 0;
     p.n_tiles = pl.n_tiles;
@@ -796,7 +922,8 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     cudaError_t err = cudaSuccess;
     if (ev_start) err = cudaEventRecord(ev_start, stream);
     // behind the threshold kernel the scan may start early; its epilogue waits for the thresholds
-    if (err == cudaSuccess) err = launch_kernel(map_q, map_bank, p, pl.grid, sp.bytes, pl.n_sample != 0 && !ev_start, stream);
+    if (err == cudaSuccess)
+        err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, pl.n_sample != 0 && !ev_start, pl.pair != 0, stream);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);
