@@ -16,11 +16,14 @@
 //              tensor-memory buffers; tcgen05.commit hands smem stages back to the
 //              producer and finished accumulators to the epilogue.
 //   warps 2-5  epilogue: thread m owns query m of the tile (= TMEM lane m).  It reads
-//              its 256 similarities of a bank tile 32 at a time, compares them with
+//              its 256 similarities of a bank tile a chunk at a time, compares them with
 //              the query's running threshold held in a register, and appends the few
 //              survivors to the query's private candidate list in global memory.
 //              When a list fills, the warp cuts it back to its best k1 with an exact
 //              radix select over registers and the threshold rises.
+//   warp 6     threshold tracker: keeps re-reading the shared histograms of the block's
+//              128 queries and posts each query's current bin threshold in shared memory,
+//              so that the epilogue threads never wait on global memory between tiles.
 //
 // A bank tile is 256 consecutive entries; the queries sit on the accumulator's
 // lanes so that the per-query threshold test costs one register compare and no
@@ -35,9 +38,9 @@
 //
 // During the full scan the blocks tighten the thresholds together.  Each query has a
 // small histogram in global memory over the similarity range above its starting
-// threshold; every survivor is counted in it, and before each bank tile a thread reads
-// its query's counters and raises its threshold to the highest bin edge that already has
-// k1 survivors at or above it.  Counters only grow, so whatever mix of old and new
+// threshold; every survivor is counted in it, the tracker warp reads the counters of the
+// block's queries over and over, and before each bank tile an epilogue thread raises its
+// threshold to the highest bin edge that was seen with k1 survivors at or above it.  Counters only grow, so whatever mix of old and new
 // values a reader sees undercounts, and a threshold derived from it still has at least
 // k1 real entries above it: the selection stays exact while the survivor rate falls
 // from k1/sample to about k1/(rows scanned so far by all blocks).
@@ -59,13 +62,15 @@ constexpr int kBlockN = 256;
 constexpr int kBlockK = 64;
 constexpr int kUmmaK = 16;
 constexpr int kMaxStages = 6;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr uint32_t kABytes = kBlockM * kBlockK * 2;  // 16 KB: a streamed slice of the query tile
 constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;  // 32 KB: a slice of a bank tile
 constexpr uint32_t kTmemCols = 512;                  // two accumulators of 256 fp32 columns
 constexpr size_t kSmemMax = 232448;                  // 227 KB of dynamic shared memory per block
-constexpr size_t kSmemFixed = 1024 + 256;            // alignment slack + barriers
+constexpr size_t kSmemFixed = 1024 + 256 + 1536;     // alignment slack + barriers + tracker mailboxes
 constexpr int kHistBins = 64;
+constexpr int kChunk = 32;                           // accumulator columns per tensor-memory load
+constexpr int kSyncTiles = 4;                        // tiles of a job whose threshold the epilogue reads itself
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
 
 // tcgen05 instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=256, M=128.
@@ -219,44 +224,59 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane: the load is asynchronous, the
-// registers hold the data only after tmem_ld_wait on the same array.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
+// kChunk consecutive fp32 columns of this thread's TMEM lane: the load is asynchronous, the
+// registers hold the data only after tmem_ld_wait on the same array (which waits for every
+// outstanding tcgen05.ld of the thread; the registers are named as in/out operands so that no
+// use of them can be scheduled ahead of the wait).
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
 }
-// Waits for every outstanding tcgen05.ld of this thread.  The registers are named as in/out
-// operands so that no use of them can be scheduled ahead of the wait.
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.wait::ld.sync.aligned;"
-        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
-          "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
-          "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
-          "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
         :
         : "memory");
 }
 
-// v[j] for a run-time j without spilling the array: a 5-level select tree.
-__device__ __forceinline__ uint32_t pick32(const uint32_t (&v)[32], int j) {
-    uint32_t a[16], b[8], c[4];
+// v[base + j] for a run-time j in [0, 16) without spilling the array: a 4-level select tree.
+template <int W>
+__device__ __forceinline__ uint32_t pick16(const uint32_t (&v)[W], int base, int j) {
+    uint32_t a[8], b[4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) a[i] = (j & 1) ? v[2 * i + 1] : v[2 * i];
+    for (int i = 0; i < 8; ++i) a[i] = (j & 1) ? v[base + 2 * i + 1] : v[base + 2 * i];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) b[i] = (j & 2) ? a[2 * i + 1] : a[2 * i];
+    for (int i = 0; i < 4; ++i) b[i] = (j & 2) ? a[2 * i + 1] : a[2 * i];
+    const uint32_t c0 = (j & 4) ? b[1] : b[0], c1 = (j & 4) ? b[3] : b[2];
+    return (j & 8) ? c1 : c0;
+}
+
+// Highest bin of a query's shared histogram with k1 counted survivors at or above it (0 when
+// there is none yet).  All sixteen loads are issued before the first is looked at.
+__device__ __forceinline__ int hist_best_bin(const unsigned *hist, int k1) {
+    uint4 c[kHistBins / 4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) c[i] = (j & 4) ? b[2 * i + 1] : b[2 * i];
-    const uint32_t d0 = (j & 8) ? c[1] : c[0], d1 = (j & 8) ? c[3] : c[2];
-    return (j & 16) ? d1 : d0;
+    for (int g = 0; g < kHistBins / 4; ++g) c[g] = __ldcg(reinterpret_cast<const uint4 *>(hist) + g);
+    int acc_cnt = 0, best = 0;
+    bool found = false;
+#pragma unroll
+    for (int g = kHistBins / 4 - 1; g >= 0; --g) {
+        const unsigned cs[4] = {c[g].x, c[g].y, c[g].z, c[g].w};
+#pragma unroll
+        for (int e = 3; e >= 0; --e) {
+            acc_cnt += (int)cs[e];
+            if (!found && acc_cnt >= k1) {
+                found = true;
+                best = g * 4 + e;
+            }
+        }
+    }
+    return best;
 }
 
 // ---- warp-wide exact selection over one candidate list ------------------------
@@ -354,6 +374,13 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // bars[0..6) full, [6..12) empty, [12..14) tmem_full, [14..16) tmem_empty, [16] queries resident
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 5);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    // tracker mailboxes, one per epilogue thread: the query it serves now (-1: none) going in,
+    // (query << 32 | bin threshold) coming back; epi_done counts epilogue warps that have finished
+    volatile int *epi_done = reinterpret_cast<volatile int *>(tmem_slot + 2);
+    volatile int *tile_seq = reinterpret_cast<volatile int *>(tmem_slot + 3);   // accumulators examined so far
+    volatile int *slot_q = reinterpret_cast<volatile int *>(reinterpret_cast<unsigned char *>(bars) + 256);
+    volatile unsigned long long *slot_tau =
+        reinterpret_cast<volatile unsigned long long *>(reinterpret_cast<unsigned char *>(bars) + 256 + 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long wait_limit = p.stall ? kTimeoutCycles / 16 : kTimeoutCycles;
@@ -372,8 +399,14 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             mbar_init(tempty0 + 8 * b, kPair ? 8 : 4);  // one arrival per epilogue warp of every block on the tile
         }
         *abort_flag = 0;
+        *epi_done = 0;
+        *tile_seq = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + kBlockM) {
+        slot_q[threadIdx.x - 64] = -1;
+        slot_tau[threadIdx.x - 64] = ~0ull;
     }
     if (warp == 0) {
         __syncwarp();
@@ -463,7 +496,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ===== epilogue: thread = one query of the tile = one TMEM lane =====
         // The thresholds, the histogram and the candidate lists belong to the kernels before this
         // one; loads and MMAs of the first tiles run ahead while the epilogue waits for them.
@@ -501,120 +534,185 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 tau_sim = key_sim_floor;
             }
+            slot_q[m] = my_hist ? q : -1;   // the tracker follows this query from now on
             int cnt = 0;
             uint64_t *my_buf = p.cand + ((size_t)list_job * kBlockM + m) * kMmaCandCap;
+            // Files one similarity that reached tau_sim.
+            auto file = [&](float s, int64_t row) {
+                if (row < p.size) {
+                    const uint64_t key = make_key(s, (int32_t)row);
+                    int bin = 0;
+                    if (my_hist) {
+                        bin = (int)floorf((s - h_lo) * h_scale);
+                        bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
+                    }
+                    if (key > tau_key && bin >= tau_bin) {
+                        my_buf[cnt++] = key;
+                        if (my_hist) atomicAdd(my_hist + bin, 1u);
+                    }
+                }
+            };
+            // One chunk of columns: store it (dense mode) or file the entries that pass the filters.
+            auto process = [&](uint32_t (&v)[kChunk], int64_t row0, int c0) {
+                if (p.mode == 1) {
+                    if (q_valid) {
+                        float4 *dst = reinterpret_cast<float4 *>(p.dense + (size_t)q * p.dense_ld + row0 + c0);
+#pragma unroll
+                        for (int j = 0; j < kChunk / 4; ++j)
+                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    }
+                    return;
+                }
+                // maxima of the 16-column groups first: nearly every group fails the test as a whole
+                constexpr int kGroups = kChunk / 16;
+                float mx[kGroups];
+#pragma unroll
+                for (int g = 0; g < kGroups; ++g) {
+                    mx[g] = __uint_as_float(v[16 * g]);
+#pragma unroll
+                    for (int j = 1; j < 16; ++j) mx[g] = fmaxf(mx[g], __uint_as_float(v[16 * g + j]));
+                }
+                float mx_all = mx[0];
+#pragma unroll
+                for (int g = 1; g < kGroups; ++g) mx_all = fmaxf(mx_all, mx[g]);
+                if (mx_all >= tau_sim) {
+#pragma unroll
+                    for (int g = 0; g < kGroups; ++g) {
+                        if (mx[g] >= tau_sim) {
+                            uint32_t pass = 0;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                pass |= (__uint_as_float(v[16 * g + j]) >= tau_sim ? 1u : 0u) << j;
+                            while (pass) {
+                                const int j = __ffs(pass) - 1;
+                                pass &= pass - 1;
+                                file(__uint_as_float(pick16(v, 16 * g, j)), row0 + c0 + 16 * g + j);
+                            }
+                        }
+                    }
+                }
+                // lists that could overflow on the next chunk are cut back to their best k1
+                uint32_t need = __ballot_sync(0xffffffffu, cnt > kMmaCandCap - kChunk);
+                while (need) {
+                    const int owner = __ffs(need) - 1;
+                    need &= need - 1;
+                    const int n = __shfl_sync(0xffffffffu, cnt, owner);
+                    uint64_t *buf = reinterpret_cast<uint64_t *>(
+                        __shfl_sync(0xffffffffu, (unsigned long long)my_buf, owner));
+                    __syncwarp();
+                    const uint64_t kth = warp_select_topk(buf, n, p.k1);
+                    if (lane == owner) {
+                        cnt = p.k1;
+                        tau_key = kth;
+                        key_sim_floor = key_sim(kth);
+                        tau_sim = fmaxf(tau_sim, key_sim_floor);
+                    }
+                }
+            };
+            auto raise_bin = [&](int best) {
+                if (best > tau_bin) {
+                    tau_bin = best;
+                    // a similarity in bin b is at least h_lo + b / h_scale up to rounding; stay a
+                    // hundredth of a bin below that and let the bin test decide
+                    tau_sim = fmaxf(key_sim_floor, h_lo + ((float)tau_bin - 0.01f) / h_scale);
+                }
+            };
+            // Takes the tracker's latest word for this query.
+            auto refresh = [&]() {
+                if (my_hist) {
+                    const unsigned long long word = slot_tau[m];
+                    if ((int)(word >> 32) == q) raise_bin((int)(uint32_t)word);
+                }
+            };
+            int sync_left = kSyncTiles;
             for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                 if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
                 tc_fence_after();
+                if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
+                // At the start of a job a threshold moves with every tile and the tracker's word comes
+                // a tile late: there the thread reads its counters itself, later it takes the word.
+                if (sync_left > 0) {
+                    --sync_left;
+                    if (my_hist) raise_bin(hist_best_bin(my_hist, p.k1));
+                } else {
+                    refresh();
+                }
                 const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
                 const int64_t row0 = (int64_t)t * kBlockN;
-                if (my_hist) {
-                    // highest bin with k1 counted survivors at or above it
-                    int acc_cnt = 0, best = 0;
-                    bool found = false;
-#pragma unroll
-                    for (int g = kHistBins / 4 - 1; g >= 0; --g) {
-                        const uint4 c = __ldcg(reinterpret_cast<const uint4 *>(my_hist) + g);
-                        const unsigned cs[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-                        for (int e = 3; e >= 0; --e) {
-                            acc_cnt += (int)cs[e];
-                            if (!found && acc_cnt >= p.k1) {
-                                found = true;
-                                best = g * 4 + e;
-                            }
-                        }
-                    }
-                    if (best > tau_bin) {
-                        tau_bin = best;
-                        // a similarity in bin b is at least h_lo + b / h_scale up to rounding; stay a
-                        // hundredth of a bin below that and let the bin test decide
-                        tau_sim = fmaxf(key_sim_floor, h_lo + ((float)tau_bin - 0.01f) / h_scale);
-                    }
-                }
-                // One 32-column chunk: store it (dense mode) or file the entries that pass the filters.
-                auto process = [&](uint32_t (&v)[32], int c0) {
-                    if (p.mode == 1) {
-                        if (q_valid) {
-                            float4 *dst = reinterpret_cast<float4 *>(p.dense + (size_t)q * p.dense_ld + row0 + c0);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                        }
-                        return;
-                    }
-                    float mx = __uint_as_float(v[0]);
-#pragma unroll
-                    for (int j = 1; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(v[j]));
-                    if (mx >= tau_sim) {
-                        uint32_t pass = 0;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) pass |= (__uint_as_float(v[j]) >= tau_sim ? 1u : 0u) << j;
-                        while (pass) {
-                            const int j = __ffs(pass) - 1;
-                            pass &= pass - 1;
-                            const float s = __uint_as_float(pick32(v, j));
-                            const int64_t row = row0 + c0 + j;
-                            if (row < p.size) {
-                                const uint64_t key = make_key(s, (int32_t)row);
-                                int bin = 0;
-                                if (my_hist) {
-                                    bin = (int)floorf((s - h_lo) * h_scale);
-                                    bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
-                                }
-                                if (key > tau_key && bin >= tau_bin) {
-                                    my_buf[cnt++] = key;
-                                    if (my_hist) atomicAdd(my_hist + bin, 1u);
-                                }
-                            }
-                        }
-                    }
-                    // lists that could overflow on the next 32 columns are cut back to their best k1
-                    uint32_t need = __ballot_sync(0xffffffffu, cnt > kMmaCandCap - 32);
-                    while (need) {
-                        const int owner = __ffs(need) - 1;
-                        need &= need - 1;
-                        const int n = __shfl_sync(0xffffffffu, cnt, owner);
-                        uint64_t *buf = reinterpret_cast<uint64_t *>(
-                            __shfl_sync(0xffffffffu, (unsigned long long)my_buf, owner));
-                        __syncwarp();
-                        const uint64_t kth = warp_select_topk(buf, n, p.k1);
-                        if (lane == owner) {
-                            cnt = p.k1;
-                            tau_key = kth;
-                            key_sim_floor = key_sim(kth);
-                            tau_sim = fmaxf(tau_sim, key_sim_floor);
-                        }
-                    }
-                };
                 // two register buffers: the next chunk's load is in flight while one is examined
-                uint32_t va[32], vb[32];
-                tmem_ld32_issue(t_addr, va);
+                uint32_t va[kChunk], vb[kChunk];
+                tmem_ld_issue(t_addr, va);
                 tmem_ld_wait(va);
 #pragma unroll 1
-                for (int c0 = 0; c0 < kBlockN; c0 += 64) {
-                    tmem_ld32_issue(t_addr + c0 + 32, vb);
-                    process(va, c0);
+                for (int c0 = 0; c0 < kBlockN - 2 * kChunk; c0 += 2 * kChunk) {
+                    tmem_ld_issue(t_addr + c0 + kChunk, vb);
+                    process(va, row0, c0);
                     tmem_ld_wait(vb);
-                    if (c0 + 64 < kBlockN) tmem_ld32_issue(t_addr + c0 + 64, va);
-                    process(vb, c0 + 32);
-                    if (c0 + 64 < kBlockN) tmem_ld_wait(va);
+                    tmem_ld_issue(t_addr + c0 + 2 * kChunk, va);
+                    refresh();
+                    process(vb, row0, c0 + kChunk);
+                    tmem_ld_wait(va);
                 }
+                tmem_ld_issue(t_addr + kBlockN - kChunk, vb);
+                process(va, row0, kBlockN - 2 * kChunk);
+                tmem_ld_wait(vb);
+                // every column of this accumulator is in registers: hand it back before the last look
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
                     if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * acc, 0)); else mbar_arrive(tempty0 + 8 * acc);
                 }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                process(vb, row0, kBlockN - kChunk);
             }
             if (p.mode == 0 && ok && qt < p.n_qt) p.cand_cnt[(size_t)list_job * kBlockM + m] = cnt;
         }
+        slot_q[m] = -1;
         if (!ok && p.mode == 0) {
             // aborting: whatever this block was to deliver counts as empty, so the merge reads nothing stale
             for (int job = worker; job < n_jobs; job += n_workers) {
                 const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
                 if (qt < p.n_qt) p.cand_cnt[((size_t)qt * p.splits + job % p.splits) * kBlockM + m] = 0;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) atomicAdd(const_cast<int *>(epi_done), 1);
+    } else {
+        // ===== threshold tracker: lane l looks after epilogue threads l, l+32, l+64, l+96 =====
+        // The counters are read on a thinning schedule: after every tile at the start of a job,
+        // where a threshold still moves with each tile, then about every eighth of the tiles done
+        // so far (the survivor rate falls like 1 / rows scanned, so a threshold that is an eighth
+        // of the scan old lets through an eighth more).  Reading them after every tile throughout
+        // costs a tenth of the kernel's time: the reads of all blocks meet the survivors' atomic
+        // updates on the same L2 lines.
+        if (p.mode == 0 && p.tau0 != nullptr) {
+            pdl_wait();
+            const long long t0 = clock64();
+            int seen = -1, job_start = 0, next_poll = 0, q_first = -2;
+            auto running = [&]() { return *epi_done < 4 && !*abort_flag && clock64() - t0 < 2 * wait_limit; };
+            while (running()) {
+                while (*tile_seq == seen && running()) __nanosleep(100);
+                seen = *tile_seq;
+                // a new job (other queries on the mailboxes) starts the schedule afresh
+                const int q_now = __shfl_sync(0xffffffffu, slot_q[lane], 0);
+                if (q_now != q_first) {
+                    q_first = q_now;
+                    job_start = seen;
+                    next_poll = seen + kSyncTiles - 1;   // until then the epilogue reads the counters itself
+                }
+                if (seen < next_poll) continue;
+                next_poll = seen + 1 + (seen - job_start) / 8;
+#pragma unroll 1
+                for (int r = 0; r < kBlockM / 32; r += 2) {
+                    const int m0 = r * 32 + lane, m1 = m0 + 32;
+                    const int q0 = slot_q[m0], q1 = slot_q[m1];
+                    // two queries at a time, so that their loads overlap
+                    const int b0 = hist_best_bin(p.hist + (size_t)(q0 < 0 ? 0 : q0) * kHistBins, p.k1);
+                    const int b1 = hist_best_bin(p.hist + (size_t)(q1 < 0 ? 0 : q1) * kHistBins, p.k1);
+                    if (q0 >= 0) slot_tau[m0] = ((unsigned long long)(uint32_t)q0 << 32) | (uint32_t)b0;
+                    if (q1 >= 0) slot_tau[m1] = ((unsigned long long)(uint32_t)q1 << 32) | (uint32_t)b1;
+                }
             }
         }
     }
