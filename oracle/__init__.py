@@ -56,6 +56,8 @@ def _load():
     lib.evk_oracle_phase1.restype = c_i32
     lib.evk_oracle_phase2.argtypes = [p, p, c_i32, p, c_f64, c_i32, p, p]
     lib.evk_oracle_phase2.restype = c_i32
+    lib.evk_oracle_phase2_zscore.argtypes = [p, p, c_i32, p, c_f64, c_i32, p, p]
+    lib.evk_oracle_phase2_zscore.restype = c_i32
     lib.evk_oracle_q_update_f64.argtypes = [p, p, p, c_i64, c_f64]
     lib.evk_oracle_q_update_f64.restype = None
     lib.evk_oracle_q_update_f32.argtypes = [p, p, p, c_i64, c_f32]
@@ -71,6 +73,8 @@ def _load():
     lib.evk_oracle_explore.argtypes = [p, p, c_i32, p, c_f64, c_i32, c_f32, ctypes.c_uint64, ctypes.c_uint64,
                                        ctypes.c_uint32, p, p]
     lib.evk_oracle_explore.restype = c_i32
+    lib.evk_oracle_explore_zscore.argtypes = lib.evk_oracle_explore.argtypes
+    lib.evk_oracle_explore_zscore.restype = c_i32
     lib.evk_oracle_q_update_decay_f64.argtypes = [p, p, p, p, c_i64]
     lib.evk_oracle_q_update_decay_f64.restype = None
     lib.evk_oracle_q_update_decay_f32.argtypes = [p, p, p, p, c_i64]
@@ -137,8 +141,9 @@ def phase1(bank_bits, query_bits, k1: int):
     return ids, sm
 
 
-def phase2(pool_ids, pool_sims, q_stage, w: float, k2: int):
-    """Cut each pool to k2 by (1-w)*sim + w*Q (score desc, sim desc, id asc)."""
+def phase2(pool_ids, pool_sims, q_stage, w: float, k2: int, zscore: bool = False):
+    """Cut each pool to k2 by (1-w)*sim + w*Q (score desc, sim desc, id asc); with zscore the
+    two terms are first replaced by their z-scores over the pool."""
     pool_ids = _c(pool_ids, np.int32)
     pool_sims = _c(pool_sims, np.float64)
     q_stage = _c(q_stage, np.float32)
@@ -148,16 +153,16 @@ def phase2(pool_ids, pool_sims, q_stage, w: float, k2: int):
     ids = np.empty((b, k2), dtype=np.int32)
     sc = np.empty((b, k2), dtype=np.float64)
     lib = _load()
+    fn = lib.evk_oracle_phase2_zscore if zscore else lib.evk_oracle_phase2
     for i in range(b):
-        lib.evk_oracle_phase2(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage),
-                              float(w), k2, _ptr(ids[i]), _ptr(sc[i]))
+        fn(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage), float(w), k2, _ptr(ids[i]), _ptr(sc[i]))
     return ids, sc
 
 
-def retrieve(bank_bits, query_bits, q_stage, k1: int, k2: int, w: float):
+def retrieve(bank_bits, query_bits, q_stage, k1: int, k2: int, w: float, zscore: bool = False):
     """Both phases; returns (ids, scores, pool_ids, pool_sims)."""
     pool_ids, pool_sims = phase1(bank_bits, query_bits, k1)
-    ids, sc = phase2(pool_ids, pool_sims, q_stage, w, k2)
+    ids, sc = phase2(pool_ids, pool_sims, q_stage, w, k2, zscore)
     return ids, sc, pool_ids, pool_sims
 
 
@@ -224,7 +229,7 @@ def philox4x32_10(counter, key) -> np.ndarray:
 
 
 def explore(pool_ids, pool_sims, q_stage, w: float, k2: int, epsilon: float, seed: int, step: int,
-            first_query: int = 0):
+            first_query: int = 0, zscore: bool = False):
     """Epsilon-greedy choice per query over canonical pools; returns (ids, scores, explored)."""
     pool_ids = _c(pool_ids, np.int32)
     pool_sims = _c(pool_sims, np.float64)
@@ -236,8 +241,9 @@ def explore(pool_ids, pool_sims, q_stage, w: float, k2: int, epsilon: float, see
     sc = np.empty((b, k2), dtype=np.float64)
     explored = np.zeros(b, dtype=np.uint8)
     lib = _load()
+    fn = lib.evk_oracle_explore_zscore if zscore else lib.evk_oracle_explore
     for i in range(b):
-        explored[i] = lib.evk_oracle_explore(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage), float(w), k2,
+        explored[i] = fn(_ptr(pool_ids[i]), _ptr(pool_sims[i]), k1, _ptr(q_stage), float(w), k2,
                                              float(np.float32(epsilon)), int(seed), int(step), first_query + i,
                                              _ptr(ids[i]), _ptr(sc[i]))
     return ids, sc, explored

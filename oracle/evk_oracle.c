@@ -16,7 +16,8 @@
  * invariants, library routines and brute force; none is "parity unpinned" except
  * the general mixing weight 0 < w < 1 of evk_oracle_phase2, whose formula is a
  * reading (the paper's own rule is w = 1) and is pinned only through its special
- * cases, a hand-worked exact example and monotonicity.
+ * cases, a hand-worked exact example and monotonicity, and the pool z-score
+ * variant evk_oracle_phase2_zscore, which the paper does not have at all.
  */
 #include <math.h>
 #include <stdint.h>
@@ -141,6 +142,69 @@ int32_t evk_oracle_phase2(const int32_t *pool_ids, const double *pool_sims, int3
     int32_t n_out = n < k2 ? n : k2;
     for (int32_t j = 0; j < k2; ++j) { ids_out[j] = -1; scores_out[j] = -INFINITY; }
     for (int32_t j = 0; j < n_out; ++j) { ids_out[j] = r[j].id; scores_out[j] = r[j].key; }
+    free(r);
+    return n_out;
+}
+
+/* Pool z-scores: a variant of the value filter with no counterpart in the paper (which
+ * normalises rewards, not scores).  Over the valid entries of ONE query's pool, each term
+ * is replaced by its z-score, z(x) = (x - mean) / std with the population standard
+ * deviation, z = 0 where std <= 1e-6; then score = (1-w)*z(sim) + w*z(Q_stage[id]).
+ * Writes the n valid entries' scores, in pool order, to scores[]; returns n. */
+static int32_t zscore_pool_scores(const int32_t *pool_ids, const double *pool_sims, int32_t k1,
+                                  const float *q_stage, double w, double *scores) {
+    int32_t n = 0;
+    double mean_s = 0.0, mean_q = 0.0, var_s = 0.0, var_q = 0.0;
+    for (int32_t j = 0; j < k1; ++j) {
+        if (pool_ids[j] < 0) continue;
+        mean_s += pool_sims[j];
+        mean_q += (double)q_stage[pool_ids[j]];
+        ++n;
+    }
+    if (n == 0) return 0;
+    mean_s /= n;
+    mean_q /= n;
+    for (int32_t j = 0; j < k1; ++j) {
+        if (pool_ids[j] < 0) continue;
+        const double ds = pool_sims[j] - mean_s, dq = (double)q_stage[pool_ids[j]] - mean_q;
+        var_s += ds * ds;
+        var_q += dq * dq;
+    }
+    const double sd_s = sqrt(var_s / n), sd_q = sqrt(var_q / n);
+    int32_t m = 0;
+    for (int32_t j = 0; j < k1; ++j) {
+        if (pool_ids[j] < 0) continue;
+        const double zs = sd_s > 1e-6 ? (pool_sims[j] - mean_s) / sd_s : 0.0;
+        const double zq = sd_q > 1e-6 ? ((double)q_stage[pool_ids[j]] - mean_q) / sd_q : 0.0;
+        scores[m++] = (1.0 - w) * zs + w * zq;
+    }
+    return n;
+}
+
+/* evk_oracle_phase2 with pool z-scores in place of the raw terms; same order rule and
+ * padding.  "Parity unpinned" as a formula (it is this library's variant); pinned through
+ * what z-scoring fixes: zero mean and unit variance over the pool, invariance under a
+ * positive affine change of Q, the orders at w = 0 and w = 1, a hand-worked example and
+ * scipy's zscore. */
+int32_t evk_oracle_phase2_zscore(const int32_t *pool_ids, const double *pool_sims, int32_t k1,
+                                 const float *q_stage, double w, int32_t k2,
+                                 int32_t *ids_out, double *scores_out) {
+    ranked_t *r = (ranked_t *)malloc((size_t)(k1 > 0 ? k1 : 1) * sizeof(ranked_t));
+    double *sc = (double *)malloc((size_t)(k1 > 0 ? k1 : 1) * sizeof(double));
+    const int32_t n = zscore_pool_scores(pool_ids, pool_sims, k1, q_stage, w, sc);
+    int32_t m = 0;
+    for (int32_t j = 0; j < k1; ++j) {
+        if (pool_ids[j] < 0) continue;
+        r[m].key = sc[m];
+        r[m].key2 = pool_sims[j];
+        r[m].id = pool_ids[j];
+        ++m;
+    }
+    qsort(r, (size_t)n, sizeof(ranked_t), ranked_cmp);
+    int32_t n_out = n < k2 ? n : k2;
+    for (int32_t j = 0; j < k2; ++j) { ids_out[j] = -1; scores_out[j] = -INFINITY; }
+    for (int32_t j = 0; j < n_out; ++j) { ids_out[j] = r[j].id; scores_out[j] = r[j].key; }
+    free(sc);
     free(r);
     return n_out;
 }
@@ -279,6 +343,37 @@ int32_t evk_oracle_explore(const int32_t *pool_ids, const double *pool_sims, int
         scores_out[i] = (1.0 - w) * pool_sims[pos] + w * (double)q_stage[pool_ids[pos]];
     }
     free(perm);
+    return 1;
+}
+
+/* evk_oracle_explore with pool z-scores: the same draws, scores from zscore_pool_scores. */
+int32_t evk_oracle_explore_zscore(const int32_t *pool_ids, const double *pool_sims, int32_t k1,
+                                  const float *q_stage, double w, int32_t k2, float epsilon,
+                                  uint64_t seed, uint64_t step, uint32_t query,
+                                  int32_t *ids_out, double *scores_out) {
+    int32_t n = 0;
+    while (n < k1 && pool_ids[n] >= 0) ++n;
+    const float u = (float)(explore_word(seed, step, query, 0) >> 8) * (1.0f / 16777216.0f);
+    if (!(u < epsilon) || n == 0) {
+        evk_oracle_phase2_zscore(pool_ids, pool_sims, k1, q_stage, w, k2, ids_out, scores_out);
+        return 0;
+    }
+    double *sc = (double *)malloc((size_t)k1 * sizeof(double));
+    zscore_pool_scores(pool_ids, pool_sims, n, q_stage, w, sc);  /* the first n slots are the valid ones */
+    int32_t *perm = (int32_t *)malloc((size_t)n * sizeof(int32_t));
+    for (int32_t i = 0; i < n; ++i) perm[i] = i;
+    const int32_t m = k2 < n ? k2 : n;
+    for (int32_t j = 0; j < k2; ++j) { ids_out[j] = -1; scores_out[j] = -INFINITY; }
+    for (int32_t i = 0; i < m; ++i) {
+        const uint32_t r = explore_word(seed, step, query, (uint32_t)(i + 1));
+        const int32_t pick = i + (int32_t)(((uint64_t)r * (uint64_t)(n - i)) >> 32);
+        const int32_t tmp = perm[i]; perm[i] = perm[pick]; perm[pick] = tmp;
+        const int32_t pos = perm[i];
+        ids_out[i] = pool_ids[pos];
+        scores_out[i] = sc[pos];
+    }
+    free(perm);
+    free(sc);
     return 1;
 }
 
