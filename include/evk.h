@@ -54,6 +54,8 @@ enum { EVK_DTYPE_F32 = 0, EVK_DTYPE_BF16 = 1 };
 enum { EVK_STAGE_DRAFT = 0, EVK_STAGE_REFINE = 1, EVK_STAGE_ALL = -1 };
 /* Which phase-1 kernel evk_retrieve uses. */
 enum { EVK_SCORING_AUTO = 0, EVK_SCORING_STREAM = 1, EVK_SCORING_TENSOR = 2 };
+/* How phase 2 mixes similarity and value (evk_mem_set_score_norm). */
+enum { EVK_NORM_NONE = 0, EVK_NORM_POOL_ZSCORE = 1 };
 
 enum { EVK_MAX_K1 = 1024, EVK_MAX_D = 2048, EVK_MAX_STAGES = 8 };
 
@@ -92,6 +94,21 @@ int64_t evk_mem_size(const evk_mem *mem);
  * STREAM forces the streaming kernel, TENSOR the tcgen05 kernel (retrieve then
  * returns EVK_ERR_UNSUPPORTED for shapes that kernel cannot take). */
 int evk_mem_set_scoring(evk_mem *mem, int mode);
+
+/* Choose how phase 2 mixes the two terms of its score.  The method ranks the pool by
+ * Q_stage alone (Section 3.2) and normalises rewards only (Section 3.4), so neither mode
+ * has a counterpart in the paper beyond w = 1 and w = 0:
+ *   EVK_NORM_NONE (default)   score = (1-w)*sim + w*Q_stage[id];
+ *   EVK_NORM_POOL_ZSCORE      each term is first replaced, per query, by its z-score over
+ *                             the query's pool: z(x) = (x - mean) / std with the population
+ *                             standard deviation of the pool's valid entries, and z = 0 for
+ *                             a column whose std is <= 1e-6.  score = (1-w)*z(sim) + w*z(Q).
+ *                             Statistics are taken in fp64, the score is rounded to fp32.
+ * The order of the result is unchanged for w = 0 and w = 1 and under any positive affine
+ * change of the value table.  Applies to evk_retrieve, evk_retrieve_host and
+ * evk_retrieve_explore; evk_merge_shards always mixes raw terms.
+ * Errors: EVK_ERR_INVALID for an unknown mode. */
+int evk_mem_set_score_norm(evk_mem *mem, int mode);
 
 /* Append n entries: M <- M ∪ {new items} (Eq. 1).  `emb` is [n][d] row-major,
  * fp32 (rounded to bf16, nearest-even) or bf16 (copied).  Entry ids are the

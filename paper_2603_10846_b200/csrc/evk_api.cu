@@ -16,6 +16,7 @@ struct evk_mem {
     uint32_t *visits;     // [n_stages][capacity] updates received (decreasing step size)
     int32_t *status;      // device status word
     int scoring;
+    int score_norm;       // EVK_NORM_*: how phase 2 mixes similarity and value
     int stall_next;       // evk_mem_inject_stall: the next tensor-path retrieve starves its consumer
     int64_t launches;
     cudaEvent_t prof_start, prof_stop;  // armed by evk_mem_profile_scoring for one retrieve
@@ -116,6 +117,7 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     m->visits = reinterpret_cast<uint32_t *>(base + l.visits);
     m->status = reinterpret_cast<int32_t *>(base + l.status);
     m->scoring = EVK_SCORING_AUTO;
+    m->score_norm = EVK_NORM_NONE;
     m->stall_next = 0;
     m->launches = 0;
     m->prof_start = m->prof_stop = nullptr;
@@ -141,6 +143,12 @@ int64_t evk_launch_count(const evk_mem *mem) { return mem ? mem->launches : 0; }
 int evk_mem_inject_stall(evk_mem *mem) {
     if (!mem) return EVK_ERR_INVALID;
     mem->stall_next = 1;
+    return EVK_OK;
+}
+
+int evk_mem_set_score_norm(evk_mem *mem, int mode) {
+    if (!mem || (mode != EVK_NORM_NONE && mode != EVK_NORM_POOL_ZSCORE)) return EVK_ERR_INVALID;
+    mem->score_norm = mode;
     return EVK_OK;
 }
 
@@ -240,8 +248,8 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     if (err == cudaSuccess)
         err = launch_merge_rerank(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect, mem->status,
                                   pool_ids_out, pool_sims_out, k2,
-                                  mem->q_tables + (size_t)stage * mem->cfg.capacity, w, ids_out, scores_out,
-                                  stream, &launches);
+                                  mem->q_tables + (size_t)stage * mem->cfg.capacity, w, mem->score_norm, ids_out,
+                                  scores_out, stream, &launches);
     mem->launches += launches;
     return cuda_status(err);
 }
@@ -458,7 +466,7 @@ int evk_retrieve_explore(evk_mem *mem, const void *queries, int q_dtype, int32_t
     if (rc != EVK_OK) return rc;
     int launches = 0;
     cudaError_t err = launch_explore(pool_ids, pool_sims, B, k1, k2, mem->q_tables + (size_t)stage * mem->cfg.capacity,
-                                     w, epsilon, seed, step, ids_out, scores_out, explored_out,
+                                     w, mem->score_norm, epsilon, seed, step, ids_out, scores_out, explored_out,
                                      static_cast<cudaStream_t>(stream), &launches);
     mem->launches += launches;
     return cuda_status(err);

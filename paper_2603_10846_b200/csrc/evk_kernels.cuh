@@ -62,11 +62,11 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
 // expect: entries every query must at least have (min(k1, size)); fewer sets EVK_ERR_INCOMPLETE.
 constexpr int kMergeMaxParts = 2048;
 // Merges each query's lists into its pool (optionally written to pool_*_user, [B][k1]) and
-// runs phase 2 on it: ids_out / scores_out [B][k2].
+// runs phase 2 on it: ids_out / scores_out [B][k2].  norm: 0 raw mix, 1 pool z-scores.
 cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
                                 int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
                                 int32_t *pool_ids_user, float *pool_sims_user,
-                                int k2, const float *q_stage, float w, int32_t *ids_out, float *scores_out,
+                                int k2, const float *q_stage, float w, int norm, int32_t *ids_out, float *scores_out,
                                 cudaStream_t stream, int *launches);
 
 // ---- Eq. 4 update -----------------------------------------------------------
@@ -84,7 +84,7 @@ cudaError_t launch_q_update_static(float *q_stage, int64_t size, const int32_t *
 
 // ---- epsilon-greedy exploration over the pool -----------------------------------------
 cudaError_t launch_explore(const int32_t *pool_ids, const float *pool_sims, int B, int k1, int k2,
-                           const float *q_stage, float w, float epsilon, uint64_t seed, uint64_t step,
+                           const float *q_stage, float w, int norm, float epsilon, uint64_t seed, uint64_t step,
                            int32_t *ids_out, float *scores_out, uint8_t *explored_out, cudaStream_t stream,
                            int *launches);
 

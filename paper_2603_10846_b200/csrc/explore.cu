@@ -44,7 +44,7 @@ struct WordStream {
 // One warp per query; lane 0 walks the partial shuffle over positions held in shared memory.
 __global__ void __launch_bounds__(32)
 explore_kernel(const int32_t *__restrict__ pool_ids, const float *__restrict__ pool_sims, int k1, int k2,
-               const float *__restrict__ q_stage, float w, float epsilon, uint64_t seed, uint64_t step,
+               const float *__restrict__ q_stage, float w, int norm, float epsilon, uint64_t seed, uint64_t step,
                int32_t *__restrict__ ids_out, float *__restrict__ scores_out, uint8_t *__restrict__ explored_out) {
     __shared__ int32_t perm[EVK_MAX_K1];
     const int q = blockIdx.x, lane = threadIdx.x;
@@ -57,6 +57,34 @@ explore_kernel(const int32_t *__restrict__ pool_ids, const float *__restrict__ p
         n += ids[i] >= 0;
     }
     n = __reduce_add_sync(0xffffffffu, n);
+    // z-score variant: pool statistics as the rerank computes them (fp64, two passes)
+    double mean_s = 0.0, mean_q = 0.0, inv_s = 0.0, inv_q = 0.0;
+    if (norm && n > 0) {
+        auto warp_sum = [](double v) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            return v;
+        };
+        double a = 0.0, b = 0.0;
+        for (int i = lane; i < k1; i += 32)
+            if (ids[i] >= 0) {
+                a += (double)sims[i];
+                b += (double)q_stage[ids[i]];
+            }
+        mean_s = warp_sum(a) / n;
+        mean_q = warp_sum(b) / n;
+        a = 0.0;
+        b = 0.0;
+        for (int i = lane; i < k1; i += 32)
+            if (ids[i] >= 0) {
+                const double ds = (double)sims[i] - mean_s, dq = (double)q_stage[ids[i]] - mean_q;
+                a += ds * ds;
+                b += dq * dq;
+            }
+        const double sd_s = sqrt(warp_sum(a) / n), sd_q = sqrt(warp_sum(b) / n);
+        inv_s = sd_s > 1e-6 ? 1.0 / sd_s : 0.0;
+        inv_q = sd_q > 1e-6 ? 1.0 / sd_q : 0.0;
+    }
     __syncwarp();
     if (lane != 0) return;
     WordStream ws(seed, step, (uint32_t)q);
@@ -77,7 +105,11 @@ explore_kernel(const int32_t *__restrict__ pool_ids, const float *__restrict__ p
             perm[pick] = tmp;
             const int pos = perm[i];
             id = ids[pos];
-            score = fmaf(w, q_stage[id], one_minus_w * sims[pos]) + 0.0f;
+            if (norm)
+                score = (float)((1.0 - (double)w) * (((double)sims[pos] - mean_s) * inv_s) +
+                                (double)w * (((double)q_stage[id] - mean_q) * inv_q)) + 0.0f;
+            else
+                score = fmaf(w, q_stage[id], one_minus_w * sims[pos]) + 0.0f;
         }
         ids_out[(size_t)q * k2 + i] = id;
         scores_out[(size_t)q * k2 + i] = score;
@@ -87,13 +119,13 @@ explore_kernel(const int32_t *__restrict__ pool_ids, const float *__restrict__ p
 }  // namespace
 
 cudaError_t launch_explore(const int32_t *pool_ids, const float *pool_sims, int B, int k1, int k2,
-                           const float *q_stage, float w, float epsilon, uint64_t seed, uint64_t step,
+                           const float *q_stage, float w, int norm, float epsilon, uint64_t seed, uint64_t step,
                            int32_t *ids_out, float *scores_out, uint8_t *explored_out, cudaStream_t stream,
                            int *launches) {
     if (B <= 0) return cudaSuccess;
     ++*launches;
     return launch_overlapped(explore_kernel, dim3(B), dim3(32), 0, stream, pool_ids, pool_sims, k1, k2, q_stage, w,
-                             epsilon, seed, step, ids_out, scores_out, explored_out);
+                             norm, epsilon, seed, step, ids_out, scores_out, explored_out);
 }
 
 }  // namespace evk

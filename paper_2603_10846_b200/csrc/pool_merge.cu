@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(kThreads)
 merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
                     int part_stride, int qt_size, int k1, int expect, int32_t *__restrict__ status,
                     int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user,
-                    int k2, const float *__restrict__ q_stage, float w,
+                    int k2, const float *__restrict__ q_stage, float w, int norm,
                     int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
     __shared__ __align__(16) uint64_t keys[kCap];
     __shared__ int offs[kMergeMaxParts + 1];
@@ -126,7 +126,7 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
     // phase 2 on the pool keys[0..n) (any order); scratch behind the pool
     uint64_t *skey = keys + EVK_MAX_K1;
     int32_t *sid = reinterpret_cast<int32_t *>(keys + 2 * EVK_MAX_K1);
-    rerank_block<kThreads>(keys, n, k2, q_stage, w, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
+    rerank_block<kThreads>(keys, n, k2, q_stage, w, norm, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
 }
 
 }  // namespace
@@ -134,14 +134,14 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
 cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
                                 int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
                                 int32_t *pool_ids_user, float *pool_sims_user,
-                                int k2, const float *q_stage, float w, int32_t *ids_out, float *scores_out,
+                                int k2, const float *q_stage, float w, int norm, int32_t *ids_out, float *scores_out,
                                 cudaStream_t stream, int *launches) {
     if (B <= 0) return cudaSuccess;
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
     ++*launches;
     return launch_overlapped(merge_rerank_kernel, dim3(B), dim3(kThreads), 0, stream, part_keys, part_counts, nparts,
                              part_stride, qt_size, k1, expect, status, pool_ids_user, pool_sims_user, k2, q_stage, w,
-                             ids_out, scores_out);
+                             norm, ids_out, scores_out);
 }
 
 }  // namespace evk

@@ -5,6 +5,11 @@
 //
 // w = 1 ranks the pool by Q_stage alone (the rule the method states); w = 0 keeps
 // the similarity order.  Results are ordered (score desc, sim desc, id asc).
+//
+// Variant (norm = 1, no counterpart in the paper, which normalises rewards only): the two
+// terms are made commensurate per query first, each as its z-score over the pool,
+//   z(x) = (x - mean_pool(x)) / std_pool(x)   (population std; 0 where the std is <= 1e-6),
+//   score = (1 - w) * z(sim) + w * z(Q_stage[id]).
 #pragma once
 
 #include "evk_common.cuh"
@@ -22,22 +27,67 @@ struct PoolEntry {
     float sim, q;
 };
 
+// Sum of v over the block, the same bits in every thread.
+template <int NT>
+__device__ double block_sum_f64(double v) {
+    __shared__ double red[NT / 32];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    __syncthreads();  // earlier readers of red are done
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int i = 0; i < NT / 32; ++i) t += red[i];
+    return t;
+}
+
+// Mean and reciprocal population std of a pool column for the z-score variant.
+struct ZStat {
+    double mean, inv_std;  // inv_std = 0 for a (nearly) constant column
+    __device__ double z(float x) const { return ((double)x - mean) * inv_std; }
+};
+constexpr double kZStdFloor = 1e-6;
+
 // Block-wide: scores the n entries that fetch(i) returns (any order), sorts them by (score
 // desc, sim desc, id asc) and writes the first k2 (padding: id -1, score -inf).
-// skey / sid: shared scratch of next_pow2(n) entries each.
+// skey / sid: shared scratch of next_pow2(n) entries each.  norm: 0 raw mix, 1 pool z-scores.
 template <int NT, class Fetch>
-__device__ void rerank_block_with(Fetch fetch, int n, int k2, float w, uint64_t *skey, int32_t *sid,
+__device__ void rerank_block_with(Fetch fetch, int n, int k2, float w, int norm, uint64_t *skey, int32_t *sid,
                                   int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
     const int tid = threadIdx.x;
     const int np2 = next_pow2(n > 1 ? n : 1);
     const float one_minus_w = 1.0f - w;
+    ZStat zs = {0.0, 0.0}, zq = {0.0, 0.0};
+    if (norm && n > 0) {
+        // two passes in fp64: means, then squared deviations
+        double a = 0.0, b = 0.0;
+        for (int i = tid; i < n; i += NT) {
+            const PoolEntry e = fetch(i);
+            a += (double)e.sim;
+            b += (double)e.q;
+        }
+        zs.mean = block_sum_f64<NT>(a) / n;
+        zq.mean = block_sum_f64<NT>(b) / n;
+        a = 0.0;
+        b = 0.0;
+        for (int i = tid; i < n; i += NT) {
+            const PoolEntry e = fetch(i);
+            a += ((double)e.sim - zs.mean) * ((double)e.sim - zs.mean);
+            b += ((double)e.q - zq.mean) * ((double)e.q - zq.mean);
+        }
+        const double sd_s = sqrt(block_sum_f64<NT>(a) / n), sd_q = sqrt(block_sum_f64<NT>(b) / n);
+        zs.inv_std = sd_s > kZStdFloor ? 1.0 / sd_s : 0.0;
+        zq.inv_std = sd_q > kZStdFloor ? 1.0 / sd_q : 0.0;
+    }
     for (int i = tid; i < np2; i += NT) {
         uint64_t key = 0;
         int32_t id = -1;  // padding compares as the largest unsigned id and a zero key: last
         if (i < n) {
             const PoolEntry e = fetch(i);
             id = e.id;
-            float score = fmaf(w, e.q, one_minus_w * e.sim);
+            float score = norm ? (float)((1.0 - (double)w) * zs.z(e.sim) + (double)w * zq.z(e.q))
+                               : fmaf(w, e.q, one_minus_w * e.sim);
             score += 0.0f;
             key = ((uint64_t)ordered_bits(score) << 32) | ordered_bits(e.sim + 0.0f);
         }
@@ -76,7 +126,7 @@ __device__ void rerank_block_with(Fetch fetch, int n, int k2, float w, uint64_t 
 // The pool as n ranking keys (similarity, id) in shared memory, values looked up in q_stage.
 template <int NT>
 __device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const float *__restrict__ q_stage, float w,
-                             uint64_t *skey, int32_t *sid, int32_t *__restrict__ ids_out,
+                             int norm, uint64_t *skey, int32_t *sid, int32_t *__restrict__ ids_out,
                              float *__restrict__ scores_out) {
     rerank_block_with<NT>(
         [=](int i) {
@@ -86,7 +136,7 @@ __device__ void rerank_block(const uint64_t *pool_keys, int n, int k2, const flo
             e.q = q_stage[e.id];
             return e;
         },
-        n, k2, w, skey, sid, ids_out, scores_out);
+        n, k2, w, norm, skey, sid, ids_out, scores_out);
 }
 
 }  // namespace evk

@@ -111,7 +111,7 @@ merge_shards_kernel(const int32_t *__restrict__ gids, const float *__restrict__ 
             e.q = qs[r];
             return e;
         },
-        n, k2, w, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
+        n, k2, w, 0, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
 }
 
 }  // namespace

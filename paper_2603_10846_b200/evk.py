@@ -34,12 +34,13 @@ EVK_ERR_INCOMPLETE = -9
 EVK_DTYPE_F32, EVK_DTYPE_BF16 = 0, 1
 EVK_STAGE_DRAFT, EVK_STAGE_REFINE, EVK_STAGE_ALL = 0, 1, -1
 EVK_SCORING_AUTO, EVK_SCORING_STREAM, EVK_SCORING_TENSOR = 0, 1, 2
+EVK_NORM_NONE, EVK_NORM_POOL_ZSCORE = 0, 1
 EVK_MAX_K1 = 1024
 
 # Every symbol include/evk.h declares.
 EXPORTS = (
     "evk_mem_bytes_required", "evk_mem_create", "evk_mem_destroy", "evk_mem_size",
-    "evk_mem_set_scoring", "evk_mem_inject_stall", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
+    "evk_mem_set_scoring", "evk_mem_set_score_norm", "evk_mem_inject_stall", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_visits_write", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
     "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
@@ -77,6 +78,7 @@ def _load() -> ctypes.CDLL:
         "evk_mem_destroy": (cint, [vp]),
         "evk_mem_size": (i64, [vp]),
         "evk_mem_set_scoring": (cint, [vp, cint]),
+        "evk_mem_set_score_norm": (cint, [vp, cint]),
         "evk_mem_inject_stall": (cint, [vp]),
         "evk_mem_insert": (cint, [vp, vp, cint, i64, cint, vp, vp, vp]),
         "evk_retrieve_workspace_bytes": (sz, [vp, i32, i32]),
@@ -182,7 +184,7 @@ class EvkMem:
 
     def __del__(self):
         h, self.handle = getattr(self, "handle", None), None
-        if h:
+        if h and _lib is not None:   # at interpreter exit the module may already be torn down
             _lib.evk_mem_destroy(h)
 
 
@@ -222,6 +224,10 @@ def evk_launch_count(mem: EvkMem) -> int:
 
 def evk_mem_set_scoring(mem: EvkMem, mode: int) -> None:
     _check(_lib.evk_mem_set_scoring(mem.handle, mode), "evk_mem_set_scoring")
+
+
+def evk_mem_set_score_norm(mem: EvkMem, mode: int) -> None:
+    _check(_lib.evk_mem_set_score_norm(mem.handle, mode), "evk_mem_set_score_norm")
 
 
 def evk_mem_insert(mem: EvkMem, emb: torch.Tensor, stage: int = EVK_STAGE_ALL,

@@ -58,8 +58,8 @@ def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0):
     return set(real.tolist()) == set(o_ids[:n_pool].tolist())
 
 
-def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, norm_scale=1.0):
-    """Phase 2 of one query, judged on the library's own pool."""
+def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, norm_scale=1.0, zscore=False):
+    """Phase 2 of one query, judged on the library's own pool.  zscore: the pool z-score variant."""
     pool_ids = np.asarray(pool_ids)
     ids = np.asarray(ids)
     scores = np.asarray(scores, dtype=np.float64)
@@ -69,7 +69,7 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
     if n_out == 0:
         return True
     sims = oracle.sims(bank_bits, query_bits)
-    o_ids, o_sc = oracle.phase2(real, sims[real], q_stage, w, real.size)   # the whole pool, ranked
+    o_ids, o_sc = oracle.phase2(real, sims[real], q_stage, w, real.size, zscore)   # the whole pool, ranked
     o_ids, o_sc = o_ids[0], o_sc[0]
     score_of = dict(zip(o_ids.tolist(), o_sc.tolist()))
     got = ids[:n_out]
@@ -77,6 +77,10 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
     assert set(got.tolist()) <= set(real.tolist()), "result id not in pool"
     want = np.array([score_of[i] for i in got.tolist()])
     scale = (1 - w) * norm_scale + w * float(np.max(np.abs(q_stage[real]))) if real.size else 1.0
+    if zscore:
+        # a similarity off by ABS * ||q|| ||e|| moves its z-score by that over the pool's std
+        sd = float(np.std(sims[real]))
+        scale = (1 - w) * norm_scale / max(sd, 1e-6) + w
     err = np.abs(scores[:n_out] - want)
     assert np.all(err <= tol(want, max(scale, 1e-30))), f"score error {err.max():.3e}"
     assert np.all(scores[:n_out][:-1] >= scores[:n_out][1:]), "result not ordered by score"
@@ -88,7 +92,7 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
     return got.tolist() == o_ids[:n_out].tolist()
 
 
-def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None, norm_scale=1.0):
+def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None, norm_scale=1.0, zscore=False):
     """out = (ids, scores, pool_ids, pool_sims) as host arrays; sample = query indices to judge."""
     ids, scores, pool_ids, pool_sims = [np.asarray(x) for x in out]
     b = queries_bits.shape[0]
@@ -98,7 +102,7 @@ def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None
     for i in sample:
         exact_pool += bool(check_pool(bank_bits, queries_bits[i], k1, pool_ids[i], pool_sims[i], norm_scale))
         exact_final += bool(check_final(bank_bits, queries_bits[i], q_stage, w, k2, pool_ids[i], ids[i],
-                                        scores[i], norm_scale))
+                                        scores[i], norm_scale, zscore))
         n += 1
     return exact_pool / max(n, 1), exact_final / max(n, 1)
 
