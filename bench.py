@@ -30,15 +30,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "retrieval queries/sec at N=1M, d=1024 bf16"
-SCAN_DRAM_BYTES_PER_ENTRY = 545.68e6 / 262224      # d = 1024: 2,081.0 B against 2,048 B algorithmic
+SCAN_DRAM_BYTES_PER_ENTRY = 542.91e6 / 262224      # d = 1024: 2,070.4 B against 2,048 B algorithmic
 UNIT = "queries/s"
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (0: about a second of them)")
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="evk", choices=["evk", "reference"])
     ap.add_argument("--workload", default="large_hbm")
     ap.add_argument("--batch", type=int, default=0, help="query batch size (0: the workload's largest)")
@@ -135,6 +135,8 @@ def run_reference(args):
     from paper_2603_10846_b200 import synth
     wl = synth.WORKLOADS[args.workload]
     b = args.batch or max(wl.batches)
+    if args.steps <= 0:
+        args.steps = 5
     bank_bits = synth.bf16_bits(synth.make_bank(wl, "cpu").to(dtype=torch.bfloat16))
     q_tab = synth.make_q_tables(wl)
     total = args.steps + args.warmup
@@ -188,6 +190,11 @@ def run_evk(args):
 
     wl = synth.WORKLOADS[args.workload]
     b = args.batch or max(wl.batches)
+    if args.steps <= 0:
+        # long enough for several clock samples: the scan of one step reads the bank once
+        # (about 6 TB/s) or does 2*B*N*d flop (about 1.2 PFLOP/s), whichever takes longer
+        est_ms = max(wl.n * wl.d * 2 / 6.0e9, 2.0 * b * wl.n * wl.d / 1.2e12) + 0.06
+        args.steps = int(min(4000, max(20, 1000.0 / est_ms)))
     n_new = 0 if wl.n < 1024 else 16           # experiences appended per step (Eq. 1)
     total_steps = args.warmup + args.steps
     capacity = wl.n + n_new * (2 * total_steps + 8)
@@ -327,7 +334,9 @@ def run_evk(args):
         value = world * b * args.steps / (elapsed_ms * 1e-3)
         e2e_value = world * b * e2e_steps / (e2e_ms * 1e-3)
         # roofline of the dominant kernel (phase-1 scoring): each launch reads the bank once
-        size = evk.evk_mem_size(mem)
+        # rows scanned by the launches that were timed (the bank grows by n_new rows per step)
+        size = wl.n + n_new * (args.warmup + (args.steps + 1) / 2.0)
+        size_end = evk.evk_mem_size(mem)             # what the retrieval-only loop scanned
         queries_per_launch = b / max(n_score_launches, 1)
         bytes_per_launch = size * wl.d * 2 + queries_per_launch * wl.d * 2
         launch_ms = statistics.mean(score_ms) / max(n_score_launches, 1)
@@ -365,8 +374,8 @@ def run_evk(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": b * wl.d * 2 + n_upd * 8,
                     "d2h_bytes_per_step": b * wl.k2 * 8, "ms_per_step": e2e_ms / e2e_steps},
             "retrieve_only": {"ms": retrieve_ms, "queries_per_s": b / (retrieve_ms * 1e-3),
-                              "bank_gbs": size * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9,
-                              "frac_of_measured_hbm": size * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                              "bank_gbs": size_end * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9,
+                              "frac_of_measured_hbm": size_end * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
         }
