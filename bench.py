@@ -194,8 +194,10 @@ def run_evk(args):
         # long enough for several clock samples: the scan of one step reads the bank once
         # (about 6 TB/s) or does 2*B*N*d flop (about 1.2 PFLOP/s), whichever takes longer
         est_ms = max(wl.n * wl.d * 2 / 6.0e9, 2.0 * b * wl.n * wl.d / 1.2e12) + 0.06
-        args.steps = int(min(4000, max(20, 1000.0 / est_ms)))
-    n_new = 0 if wl.n < 1024 else 16           # experiences appended per step (Eq. 1)
+        args.steps = int(min(2000, max(20, 1000.0 / est_ms)))
+    # experiences appended per step (Eq. 1): 16, fewer where that would grow the bank by more
+    # than about 3 % over the run (the workload's N is what the metric is quoted on)
+    n_new = 0 if wl.n < 1024 else max(1, min(16, int(0.03 * wl.n / (args.warmup + args.steps))))
     total_steps = args.warmup + args.steps
     capacity = wl.n + n_new * (2 * total_steps + 8)
 

@@ -52,11 +52,15 @@ __device__ __forceinline__ int warp_claim_slot(bool want, int *counter) {
 // same arguments; n <= NT * PER_THREAD; 0 < k < n.  Returns the k-th largest key.
 //   hist: 256 ints of shared memory; scal: 4 uint64 of shared memory.
 // ---------------------------------------------------------------------------
-template <int NT, int PER_THREAD>
+//   SKIP_COMMON: look first for the bits all keys agree on and skip their passes.  Pays when
+//   the lists are long and similar (the merge of many lists); costs a pass otherwise.
+template <int NT, int PER_THREAD, bool SKIP_COMMON = true>
 __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, uint64_t *scal) {
     const int tid = threadIdx.x;
     uint64_t prefix = 0, mask = 0;
     int kk = k;
+    uint64_t common = 0, varying = ~(uint64_t)0;
+    if constexpr (SKIP_COMMON) {
     // Bits on which all keys agree (sign and exponent of similarities in a narrow range, the
     // upper id bits of a small bank) need no pass: every key would fall into one bin, and the
     // shared-memory atomics on that single counter would run one after another.
@@ -80,9 +84,10 @@ __device__ uint64_t block_select_topk(uint64_t *keys, int n, int k, int *hist, u
         }
     }
     __syncthreads();
-    const uint64_t common = ((uint64_t)(uint32_t)hist[1] << 32) | (uint32_t)hist[0];
-    const uint64_t varying = common ^ (((uint64_t)(uint32_t)hist[3] << 32) | (uint32_t)hist[2]);
+    common = ((uint64_t)(uint32_t)hist[1] << 32) | (uint32_t)hist[0];
+    varying = common ^ (((uint64_t)(uint32_t)hist[3] << 32) | (uint32_t)hist[2]);
     __syncthreads();
+    }
     for (int shift = 56; shift >= 0; shift -= 8) {
         if (((varying >> shift) & 0xff) == 0) {
             prefix |= common & ((uint64_t)0xff << shift);

@@ -140,7 +140,7 @@ score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
         for (int q = 0; q < nq; ++q) {
             const int n = counts[q];
             if (n > cap - kRowsPerIter) {
-                const uint64_t kth = block_select_topk<kThreads, kSelPerThread>(keys + (size_t)q * cap, n, k1, hist, scal);
+                const uint64_t kth = block_select_topk<kThreads, kSelPerThread, false>(keys + (size_t)q * cap, n, k1, hist, scal);
                 if (tid == 0) {
                     counts[q] = k1;
                     tau_key[q] = kth;
@@ -154,7 +154,7 @@ score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
     for (int q = 0; q < nq; ++q) {
         int n = counts[q];
         if (n > k1) {
-            block_select_topk<kThreads, kSelPerThread>(keys + (size_t)q * cap, n, k1, hist, scal);
+            block_select_topk<kThreads, kSelPerThread, false>(keys + (size_t)q * cap, n, k1, hist, scal);
             n = k1;
         }
         const size_t list = (size_t)(q_base + q) * nparts + blockIdx.x;
@@ -201,6 +201,37 @@ cudaError_t launch_nch(int qb, const __nv_bfloat16 *bank, int64_t size, int d,
     return launch_one<1, NCH>(bank, size, d, queries, q_base, nq, k1, plan, part_keys, part_counts, stream);
 }
 
+// Blocks of this variant that fit on one SM (registers and shared memory), asked of the runtime:
+// the grid is sized to exactly one wave of them.
+template <int QB, int NCH>
+int blocks_per_sm(size_t smem) {
+    auto kern = score_stream_kernel<QB, NCH>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kThreads, smem) != cudaSuccess || n < 1) return 1;
+    return n;
+}
+
+template <int NCH>
+int blocks_per_sm_nch(int qb, size_t smem) {
+    if constexpr (NCH <= 4) {
+        if (qb == 4) return blocks_per_sm<4, NCH>(smem);
+    }
+    return qb == 2 ? blocks_per_sm<2, NCH>(smem) : blocks_per_sm<1, NCH>(smem);
+}
+
+int blocks_per_sm_for(int qb, int nch, size_t smem) {
+    switch (nch) {
+        case 1: return blocks_per_sm_nch<1>(qb, smem);
+        case 2: return blocks_per_sm_nch<2>(qb, smem);
+        case 3: return blocks_per_sm_nch<3>(qb, smem);
+        case 4: return blocks_per_sm_nch<4>(qb, smem);
+        case 6: return blocks_per_sm_nch<6>(qb, smem);
+        case 8: return blocks_per_sm_nch<8>(qb, smem);
+        default: return 1;
+    }
+}
+
 int nch_for(int d) {
     const int chunks = d / 8;
     const int need = (chunks + 31) / 32;
@@ -222,8 +253,10 @@ StreamPlan stream_plan(int64_t size, int d, int B, int k1) {
     if (p.qb > qb_max) p.qb = qb_max;
     p.cap = stream_cap(k1);
     p.smem = stream_smem(p.qb, p.cap);
-    // Registers hold the queries, so occupancy falls as qb*nch grows; 2-4 blocks per SM.
-    const int ctas_per_sm = (p.qb * nch >= 12) ? 2 : ((p.qb * nch >= 6) ? 3 : 4);
+    // Registers hold the queries, so occupancy falls as qb*nch grows (1-4 blocks per SM); a grid
+    // that is not a whole wave of resident blocks leaves a ragged second wave.
+    int ctas_per_sm = blocks_per_sm_for(p.qb, nch, p.smem);
+    if (ctas_per_sm > 4) ctas_per_sm = 4;
     int64_t iters = (size + kRowsPerIter - 1) / kRowsPerIter;
     int64_t grid = (int64_t)kNumSM * ctas_per_sm;
     if (grid > iters) grid = iters;
