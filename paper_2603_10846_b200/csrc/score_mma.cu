@@ -71,6 +71,7 @@ constexpr size_t kSmemFixed = 1024 + 256 + 1536;     // alignment slack + barrie
 constexpr int kHistBins = 64;
 constexpr int kChunk = 32;                           // accumulator columns per tensor-memory load
 constexpr int kSyncTiles = 4;                        // tiles of a job whose threshold the epilogue reads itself
+constexpr int kSyncAlways = 1 << 28;                 // ... or every tile: the tracker stays idle
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
 
 // tcgen05 instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=256, M=128.
@@ -93,6 +94,7 @@ struct MmaParams {
     float *dense;       // [B][dense_ld]
     int dense_ld;
     int32_t *status;
+    int sync_tiles;     // kSyncTiles, or kSyncAlways when the scan is bound by HBM and the epilogue has time
     int stall;          // test aid: the producer of the full scan issues no loads, so a bounded wait runs out
 };
 
@@ -625,7 +627,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if ((int)(word >> 32) == q) raise_bin((int)(uint32_t)word);
                 }
             };
-            int sync_left = kSyncTiles;
+            int sync_left = p.sync_tiles;
             for (int t = split; t < p.n_tiles && ok; t += p.splits) {
                 if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
                 tc_fence_after();
@@ -686,7 +688,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // of the scan old lets through an eighth more).  Reading them after every tile throughout
         // costs a tenth of the kernel's time: the reads of all blocks meet the survivors' atomic
         // updates on the same L2 lines.
-        if (p.mode == 0 && p.tau0 != nullptr) {
+        if (p.mode == 0 && p.tau0 != nullptr && p.sync_tiles != kSyncAlways) {
             pdl_wait();
             const long long t0 = clock64();
             int seen = -1, job_start = 0, next_poll = 0, q_first = -2;
@@ -699,7 +701,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (q_now != q_first) {
                     q_first = q_now;
                     job_start = seen;
-                    next_poll = seen + kSyncTiles - 1;   // until then the epilogue reads the counters itself
+                    next_poll = seen + p.sync_tiles - 1;   // until then the epilogue reads the counters itself
                 }
                 if (seen < next_poll) continue;
                 next_poll = seen + 1 + (seen - job_start) / 8;
@@ -733,37 +735,120 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
 }
 
-// k1-th largest of each query's sample similarities -> starting threshold.
-constexpr int kSelThreads = 512;
+// A starting threshold per query from its sample similarities: any value that at least k1 of
+// the sampled entries reach is a lower bound of the query's final k1-th similarity.  The exact
+// k1-th largest is not needed, so one pass over a fine histogram of the sample's range picks
+// the highest bin edge with k1 samples at or above it, and the threshold is the smallest
+// sample in those bins (exact whatever the rounding of the bin arithmetic).
+constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = kMmaSample / kSelThreads;
+constexpr int kSelBins = 1024;
 
 __global__ void __launch_bounds__(kSelThreads)
 sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0,
                         float2 *__restrict__ range, unsigned *__restrict__ hist_out) {
-    __shared__ uint64_t keys[kMmaSample];
-    __shared__ int hist[256];
-    __shared__ uint64_t scal[4];
-    __shared__ unsigned long long top;
-    const int q = blockIdx.x;
+    __shared__ int bins[kSelBins];
+    __shared__ float red_lo[kSelThreads / 32], red_hi[kSelThreads / 32];
+    __shared__ int red_cnt[kSelThreads / 32];
+    __shared__ int chosen;
+    const int q = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_trigger();
     pdl_wait();
-    if (threadIdx.x == 0) top = 0;
-    for (int i = threadIdx.x; i < n_sample; i += kSelThreads) keys[i] = make_key(dense[(size_t)q * ld + i], i);
-    for (int i = threadIdx.x; i < kHistBins; i += kSelThreads) hist_out[(size_t)q * kHistBins + i] = 0;
+    for (int i = tid; i < kHistBins; i += kSelThreads) hist_out[(size_t)q * kHistBins + i] = 0;
+    for (int i = tid; i < kSelBins; i += kSelThreads) bins[i] = 0;
+    if (tid == 0) chosen = 0;
+    // this thread's samples; a non-finite similarity counts as the lowest value
+    float v[kSelPerThread];
+    float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+        const int i = tid + j * kSelThreads;
+        float x = (i < n_sample) ? dense[(size_t)q * ld + i] : -INFINITY;
+        if (i < n_sample && !(fabsf(x) <= 3.0e38f)) x = -3.0e38f;
+        v[j] = x;
+        if (i < n_sample) {
+            lo = fminf(lo, x);
+            hi = fmaxf(hi, x);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+    }
+    if (lane == 0) {
+        red_lo[warp] = lo;
+        red_hi[warp] = hi;
+    }
     __syncthreads();
-    const uint64_t kth = block_select_topk<kSelThreads, kSelPerThread>(keys, n_sample, k1, hist, scal);
-    for (int i = threadIdx.x; i < k1; i += kSelThreads) atomicMax(&top, (unsigned long long)keys[i]);
+#pragma unroll
+    for (int i = 0; i < kSelThreads / 32; ++i) {
+        lo = fminf(lo, red_lo[i]);
+        hi = fmaxf(hi, red_hi[i]);
+    }
+    float scale = (float)kSelBins / (hi - lo);
+    if (!(scale > 0.0f) || !(scale < 3.0e38f)) scale = 0.0f;   // no spread: everything in bin 0
+    int my_bin[kSelPerThread];
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+        int b = (int)((v[j] - lo) * scale);
+        b = b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
+        my_bin[j] = b;
+        if (tid + j * kSelThreads < n_sample) atomicAdd(&bins[b], 1);
+    }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    // thread t owns bins [4t, 4t+4); count of samples in its bins and in all higher ones
+    int mine[4], sum = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        mine[j] = bins[4 * tid + j];
+        sum += mine[j];
+    }
+    int incl = sum;   // this lane and the higher lanes of the warp
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int u = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += u;
+    }
+    if (lane == 0) red_cnt[warp] = incl;
+    __syncthreads();
+    int above = incl - sum;   // samples in bins higher than this thread's
+    for (int i = warp + 1; i < kSelThreads / 32; ++i) above += red_cnt[i];
+    if (above < k1 && k1 <= above + sum) {   // exactly one thread: the k1-th largest lies in its bins
+        int c = above, b = 4 * tid;
+#pragma unroll
+        for (int j = 3; j >= 0; --j) {
+            if (k1 <= c + mine[j]) {
+                b = 4 * tid + j;
+                break;
+            }
+            c += mine[j];
+        }
+        chosen = b;
+    }
+    __syncthreads();
+    const int b_min = chosen;
+    float t = INFINITY;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j)
+        if (tid + j * kSelThreads < n_sample && my_bin[j] >= b_min) t = fminf(t, v[j]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t = fminf(t, __shfl_xor_sync(0xffffffffu, t, off));
+    if (lane == 0) red_lo[warp] = t;   // last read of red_lo was before two barriers
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < kSelThreads / 32; ++i) t = fminf(t, red_lo[i]);
         // the shared histogram spans from the starting threshold to half a range above the sample's
         // best similarity; whatever lies higher is counted in the last bin
-        const float lo = key_sim(kth), best = key_sim((uint64_t)top);
-        const float hi = best + 0.5f * (best - lo);
-        float scale = 0.0f;  // 0 switches the histogram off (a sample without spread)
-        if (hi - lo > 1e-2f * fmaxf(fabsf(lo), fabsf(hi)) && hi - lo > 1e-30f) scale = (float)kHistBins / (hi - lo);
-        if (!(scale > 0.0f) || !(scale < 3.0e38f)) scale = 0.0f;
-        tau0[q] = lo;
-        range[q] = make_float2(lo, scale);
+        const float start = t, best = hi;
+        const float top = best + 0.5f * (best - start);
+        float h_scale = 0.0f;  // 0 switches the histogram off (a sample without spread)
+        if (top - start > 1e-2f * fmaxf(fabsf(start), fabsf(top)) && top - start > 1e-30f)
+            h_scale = (float)kHistBins / (top - start);
+        if (!(h_scale > 0.0f) || !(h_scale < 3.0e38f)) h_scale = 0.0f;
+        tau0[q] = start;
+        range[q] = make_float2(start, h_scale);
     }
 }
 
@@ -966,6 +1051,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.tau0 = nullptr;
     p.range = range;
     p.hist = hist;
+    // One query tile: the scan runs at HBM speed, a bank tile arrives every ~11 us and the epilogue
+    // idles most of that, so it reads its counters itself before every tile (freshest thresholds).
+    // More tiles: the tensor cores set the pace and the reads move to the tracker warp.
+    p.sync_tiles = pl.pair ? kSyncTiles : kSyncAlways;
     p.a_resident = sp.a_resident;
     p.a_rows = sp.a_rows;
     p.n_stages = sp.n_stages;

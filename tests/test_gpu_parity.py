@@ -161,6 +161,7 @@ def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None, scoring=None):
     (20000, 1024, 4, 1, 1),      # k1 = k2 = 1: plain argmax
     (300, 64, 130, 16, 4),       # two query tiles, the second nearly empty; bank just over one tile
     (66000, 128, 150, 512, 32),  # sampled thresholds, two query tiles, widest pool of the tensor path
+    (40000, 128, 330, 96, 8),    # three query tiles: the second pair of blocks has one tile of queries only
 ])
 def test_edge_shapes(evk, n, d, b, k1, k2, scoring):
     _random_case(evk, n, d, b, k1, k2, 0.5, seed=n, scoring=scoring)
