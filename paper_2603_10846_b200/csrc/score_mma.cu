@@ -363,7 +363,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int n_jobs = (kPair ? (p.n_qt + 1) / 2 : p.n_qt) * p.splits;
-    const int k_chunks = p.d / kBlockK;
+    // a width that is no multiple of 64 ends in a partial slice: TMA fills the columns beyond d with
+    // zeros, which add nothing to a similarity
+    const int k_chunks = (p.d + kBlockK - 1) / kBlockK;
     // [resident query tile: k_chunks slices of a_rows x 128 B] [ring of n_stages stages] [barriers]
     const uint32_t a_slice = (uint32_t)p.a_rows * 128u;
     const uint32_t a_region = p.a_resident ? (uint32_t)k_chunks * a_slice : 0u;
@@ -892,7 +894,7 @@ struct SmemPlan {
 SmemPlan smem_plan(int B, int d) {
     SmemPlan sp;
     const int rows = B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM;
-    const size_t a_bytes = (size_t)rows * d * 2;
+    const size_t a_bytes = (size_t)rows * ((d + kBlockK - 1) / kBlockK * kBlockK) * 2;
     const size_t budget = kSmemMax - kSmemFixed;
     if (B <= kBlockM && a_bytes + 3 * (size_t)kBBytes <= budget) {
         sp.a_resident = 1;
@@ -992,7 +994,8 @@ MmaLayout mma_layout(int B) {
 }  // namespace
 
 bool mma_supported(int d, int k1) {
-    return d % kBlockK == 0 && d >= kBlockK && k1 <= kMmaCandCap / 2 && encode_fn() != nullptr;
+    // rows must start on 16-byte boundaries for TMA (d % 8 == 0) and span at least one 64-column slice
+    return d % 8 == 0 && d >= kBlockK && k1 <= kMmaCandCap / 2 && encode_fn() != nullptr;
 }
 
 MmaPlan mma_plan(int64_t size, int B, int k1) {

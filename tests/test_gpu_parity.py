@@ -26,7 +26,7 @@ def scoring(request, evk):
 
 
 def tensor_unsupported(evk, scoring, d, k1):
-    return scoring == evk.EVK_SCORING_TENSOR and (d % 64 != 0 or k1 > 512)
+    return scoring == evk.EVK_SCORING_TENSOR and (d < 64 or k1 > 512)
 
 
 def host_bits(t):
@@ -156,6 +156,7 @@ def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None, scoring=None):
     (1, 64, 3, 8, 2),            # single entry, pool mostly padding
     (37, 8, 5, 64, 64),          # bank smaller than k1, narrowest rows, k2 = k1
     (1000, 776, 7, 100, 10),     # width not a multiple of 256, ragged row count
+    (30000, 200, 140, 40, 6),    # width not a multiple of 64 (zero-filled last slice), sampled thresholds, two query tiles
     (4097, 2048, 2, 1024, 16),   # widest rows, largest pool
     (70001, 256, 9, 33, 5),      # several tiles per block plus a tail
     (20000, 1024, 4, 1, 1),      # k1 = k2 = 1: plain argmax
