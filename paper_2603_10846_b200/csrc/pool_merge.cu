@@ -68,7 +68,35 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
     __syncthreads();
     const int total = offs[nparts];
 
-    for (int base = 0; base < total; base += kBatch) {
+    if (total <= kCap) {
+        // Everything fits at once: each warp copies whole lists to their places, no search per key.
+        // Four lists per warp and step, their loads issued together; a list longer than a warp
+        // finishes in the loop behind.
+        const int warp = tid >> 5, lane = tid & 31;
+        constexpr int kWarps = kThreads / 32;
+        for (int p0 = warp; p0 < nparts; p0 += 4 * kWarps) {
+            uint64_t v[4];
+            int first[4], cnt[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int p = p0 + u * kWarps;
+                first[u] = p < nparts ? offs[p] : 0;
+                cnt[u] = p < nparts ? offs[p + 1] - first[u] : 0;
+                v[u] = lane < cnt[u] ? part_keys[(list0 + (size_t)p * qt_size) * part_stride + lane] : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (lane < cnt[u]) keys[first[u] + lane] = v[u];
+                if (cnt[u] > 32) {
+                    const uint64_t *src = part_keys + (list0 + (size_t)(p0 + u * kWarps) * qt_size) * part_stride;
+                    for (int i = 32 + lane; i < cnt[u]; i += 32) keys[first[u] + i] = src[i];
+                }
+            }
+        }
+        if (tid == 0) count = total;
+        __syncthreads();
+    }
+    for (int base = 0; base < total && total > kCap; base += kBatch) {
         const uint64_t t = tau;
 #pragma unroll
         for (int j = 0; j < kBatch / kThreads; ++j) {

@@ -48,6 +48,7 @@ struct ZStat {
     __device__ double z(float x) const { return ((double)x - mean) * inv_std; }
 };
 constexpr double kZStdFloor = 1e-6;
+constexpr int kRankByCount = 256;   // pools up to this size are ranked by counting instead of sorted
 
 // Block-wide: scores the n entries that fetch(i) returns (any order), sorts them by (score
 // desc, sim desc, id asc) and writes the first k2 (padding: id -1, score -inf).
@@ -93,6 +94,46 @@ __device__ void rerank_block_with(Fetch fetch, int n, int k2, float w, int norm,
         }
         skey[i] = key;
         sid[i] = id;
+    }
+    if (n <= kRankByCount) {
+        // A small pool is ranked by counting: every entry counts the entries that rank before it
+        // (all threads read the same entry at a time, a broadcast) and, being one of the first k2,
+        // writes itself to its place.  No barrier between steps, a fraction of the sorting network's time.
+        __syncthreads();
+        for (int i = tid; i < n; i += NT) {
+            const uint64_t ka = skey[i];
+            const int32_t ia = sid[i];
+            int rank = 0;
+            // eight entries per step, loaded together (padding entries rank behind every real one)
+            int j = 0;
+            for (; j + 8 <= np2; j += 8) {
+                uint64_t kb[8];
+                int32_t ib[8];
+#pragma unroll
+                for (int u = 0; u < 8; u += 2) {
+                    const ulonglong2 k2v = *reinterpret_cast<const ulonglong2 *>(skey + j + u);
+                    kb[u] = k2v.x;
+                    kb[u + 1] = k2v.y;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; u += 4) {
+                    const int4 i4 = *reinterpret_cast<const int4 *>(sid + j + u);
+                    ib[u] = i4.x; ib[u + 1] = i4.y; ib[u + 2] = i4.z; ib[u + 3] = i4.w;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) rank += rerank_before(kb[u], ib[u], ka, ia) ? 1 : 0;
+            }
+            for (; j < n; ++j) rank += rerank_before(skey[j], sid[j], ka, ia) ? 1 : 0;
+            if (rank < k2) {
+                ids_out[rank] = ia;
+                scores_out[rank] = from_ordered_bits((uint32_t)(ka >> 32));
+            }
+        }
+        for (int i = n + tid; i < k2; i += NT) {
+            ids_out[i] = -1;
+            scores_out[i] = -INFINITY;
+        }
+        return;
     }
     bool wide_before = true;  // stages with stride <= 32 stay inside a warp's own 64 elements
     for (int size = 2; size <= np2; size <<= 1) {
