@@ -62,6 +62,7 @@ constexpr int kBlockN = 256;
 constexpr int kBlockK = 64;
 constexpr int kUmmaK = 16;
 constexpr int kMaxStages = 6;
+constexpr int kResidentStages = 4;                   // ring depth used (more fit, fewer are slower)
 constexpr int kThreads = 224;
 constexpr uint32_t kABytes = kBlockM * kBlockK * 2;  // 16 KB: a streamed slice of the query tile
 constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;  // 32 KB: a slice of a bank tile
@@ -900,7 +901,9 @@ SmemPlan smem_plan(int B, int d) {
         sp.a_resident = 1;
         sp.a_rows = rows;
         size_t st = (budget - a_bytes) / kBBytes;
-        sp.n_stages = (int)(st > (size_t)kMaxStages ? kMaxStages : st);
+        // four stages, even where six would fit: measured 3 % faster over 2 GiB at 1-32 queries
+        // (0.318 against 0.328 ms at one query; two stages: 0.372)
+        sp.n_stages = (int)(st > (size_t)kResidentStages ? kResidentStages : st);
         sp.bytes = kSmemFixed + a_bytes + (size_t)sp.n_stages * kBBytes;
     } else {
         sp.a_resident = 0;
@@ -1102,8 +1105,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     if (pl.pair) {
         p.a_resident = 0;
         p.a_rows = kBlockM;
-        p.n_stages = kMaxStages;
-        smem_bytes = kSmemFixed + (size_t)kMaxStages * (kABytes + kBBytes / 2);
+        // four stages here too: the same speed as six on short scans, 5 % faster on the long
+        // power-capped one (19.7 against 20.7 ms for 4,096 queries over 6 GiB)
+        p.n_stages = kResidentStages;
+        smem_bytes = kSmemFixed + (size_t)kResidentStages * (kABytes + kBBytes / 2);
     }
     p.size = size;
     p.mode = 0;
