@@ -294,6 +294,24 @@ def run_evk(args):
     torch.cuda.synchronize()
     retrieve_ms = r_start.elapsed_time(r_stop) / r_iters
 
+    # ---- the value update alone (Eq. 4), one batch of the step's size per launch ----
+    if own_updates:
+        u_batches = own_updates
+    else:
+        u_batches = [(ids_out.reshape(-1).clone(), r_sets[j]) for j in range(min(4, n_batches))]
+    longest_chain = int(torch.bincount(u_batches[0][0].clamp(min=0).to(torch.int64)).max().item()) if n_upd else 0
+    u_start, u_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        evk.evk_q_update(mem, u_batches[i % len(u_batches)][0], i % 2, u_batches[i % len(u_batches)][1], wl.alpha)
+    torch.cuda.synchronize()
+    u_start.record(stream)
+    for i in range(r_iters):
+        evk.evk_q_update(mem, u_batches[i % len(u_batches)][0], i % 2, u_batches[i % len(u_batches)][1], wl.alpha)
+    u_stop.record(stream)
+    torch.cuda.synchronize()
+    update_us = 1e3 * u_start.elapsed_time(u_stop) / r_iters
+    assert evk.evk_last_status(mem) == 0
+
     # ---- end to end through the host-buffer entry points ----
     q_host = [query_sets[j % n_batches].cpu().pin_memory() for j in range(4)]
     ids_h = torch.empty((b, wl.k2), dtype=torch.int32).pin_memory()
@@ -382,6 +400,9 @@ def run_evk(args):
             "retrieve_only": {"ms": retrieve_ms, "queries_per_s": b / (retrieve_ms * 1e-3),
                               "bank_gbs": size_end * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9,
                               "frac_of_measured_hbm": size_end * wl.d * 2 / (retrieve_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "update_only": {"us_per_batch": update_us, "updates": int(n_upd),
+                            "updates_per_s": n_upd / (update_us * 1e-6) if update_us > 0 else None,
+                            "longest_duplicate_chain": longest_chain},
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
         }
