@@ -70,7 +70,7 @@ constexpr uint32_t kTmemCols = 512;                  // two accumulators of 256 
 constexpr size_t kSmemMax = 232448;                  // 227 KB of dynamic shared memory per block
 constexpr size_t kSmemFixed = 1024 + 256 + 1536;     // alignment slack + barriers + tracker mailboxes
 constexpr int kHistBins = 64;
-constexpr int kChunk = 32;                           // accumulator columns per tensor-memory load
+constexpr int kChunk = 32;                           // accumulator columns per tensor-memory load (pick() assumes 32)
 constexpr int kSyncTiles = 4;                        // tiles of a job whose threshold the epilogue reads itself
 constexpr int kSyncAlways = 1 << 28;                 // ... or every tile: the tracker stays idle
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
@@ -253,16 +253,18 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
         : "memory");
 }
 
-// v[base + j] for a run-time j in [0, 16) without spilling the array: a 4-level select tree.
-template <int W>
-__device__ __forceinline__ uint32_t pick16(const uint32_t (&v)[W], int base, int j) {
-    uint32_t a[8], b[4];
+// v[j] for a run-time j without spilling the array: a select tree, one level per bit of j.
+__device__ __forceinline__ uint32_t pick(const uint32_t (&v)[32], int j) {
+    const bool b0 = j & 1, b1 = j & 2, b2 = j & 4, b3 = j & 8, b4 = j & 16;
+    uint32_t a[16], b[8], c[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = (j & 1) ? v[base + 2 * i + 1] : v[base + 2 * i];
+    for (int i = 0; i < 16; ++i) a[i] = b0 ? v[2 * i + 1] : v[2 * i];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) b[i] = (j & 2) ? a[2 * i + 1] : a[2 * i];
-    const uint32_t c0 = (j & 4) ? b[1] : b[0], c1 = (j & 4) ? b[3] : b[2];
-    return (j & 8) ? c1 : c0;
+    for (int i = 0; i < 8; ++i) b[i] = b1 ? a[2 * i + 1] : a[2 * i];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = b2 ? b[2 * i + 1] : b[2 * i];
+    const uint32_t d0 = b3 ? c[1] : c[0], d1 = b3 ? c[3] : c[2];
+    return b4 ? d1 : d0;
 }
 
 // Highest bin of a query's shared histogram with k1 counted survivors at or above it (0 when
@@ -556,7 +558,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const uint64_t key = make_key(s, (int32_t)row);
                     int bin = 0;
                     if (my_hist) {
-                        bin = (int)floorf((s - h_lo) * h_scale);
+                        // truncation and the clamp at 0 together equal floor and the clamp
+                        bin = __float2int_rz((s - h_lo) * h_scale);
                         bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
                     }
                     if (key > tau_key && bin >= tau_bin) {
@@ -577,32 +580,31 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     }
                     return;
                 }
-                // maxima of the 16-column groups first: nearly every group fails the test as a whole
-                constexpr int kGroups = kChunk / 16;
-                float mx[kGroups];
+                // The epilogue warps run one to a scheduler, so every dependent instruction costs its full
+                // latency: the code below is written as short trees, not chains.  First the chunk's maximum
+                // (nearly every chunk fails the test as a whole), four strands of eight.
+                float mx[4];
 #pragma unroll
-                for (int g = 0; g < kGroups; ++g) {
-                    mx[g] = __uint_as_float(v[16 * g]);
+                for (int g = 0; g < 4; ++g) {
+                    mx[g] = __uint_as_float(v[g]);
 #pragma unroll
-                    for (int j = 1; j < 16; ++j) mx[g] = fmaxf(mx[g], __uint_as_float(v[16 * g + j]));
+                    for (int j = g + 4; j < kChunk; j += 4) mx[g] = fmaxf(mx[g], __uint_as_float(v[j]));
                 }
-                float mx_all = mx[0];
+                if (fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) >= tau_sim) {
+                    // one bit per column that passes, gathered by a tree of ORs
+                    uint32_t bits[kChunk];
 #pragma unroll
-                for (int g = 1; g < kGroups; ++g) mx_all = fmaxf(mx_all, mx[g]);
-                if (mx_all >= tau_sim) {
+                    for (int j = 0; j < kChunk; ++j) bits[j] = __uint_as_float(v[j]) >= tau_sim ? (1u << j) : 0u;
 #pragma unroll
-                    for (int g = 0; g < kGroups; ++g) {
-                        if (mx[g] >= tau_sim) {
-                            uint32_t pass = 0;
+                    for (int w = kChunk / 2; w >= 1; w >>= 1) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                pass |= (__uint_as_float(v[16 * g + j]) >= tau_sim ? 1u : 0u) << j;
-                            while (pass) {
-                                const int j = __ffs(pass) - 1;
-                                pass &= pass - 1;
-                                file(__uint_as_float(pick16(v, 16 * g, j)), row0 + c0 + 16 * g + j);
-                            }
-                        }
+                        for (int j = 0; j < w; ++j) bits[j] |= bits[j + w];
+                    }
+                    uint32_t pass = bits[0];
+                    while (pass) {
+                        const int j = __ffs(pass) - 1;
+                        pass &= pass - 1;
+                        file(__uint_as_float(pick(v, j)), row0 + c0 + j);
                     }
                 }
                 // lists that could overflow on the next chunk are cut back to their best k1
