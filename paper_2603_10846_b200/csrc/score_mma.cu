@@ -649,7 +649,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 // a tile late: there the thread reads its counters itself, later it takes the word.
                 if (sync_left > 0) {
                     --sync_left;
-                    if (my_hist) raise_bin(hist_best_bin(my_hist, p.k1));
+                    // (nothing to read before the block's very first tile: every block starts at once
+                    // and the counters are still empty)
+                    if (my_hist && !(job == worker && t == split)) raise_bin(hist_best_bin(my_hist, p.k1));
                 } else {
                     refresh();
                 }
