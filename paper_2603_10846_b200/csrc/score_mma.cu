@@ -3,27 +3,33 @@
 // tensor memory), with the top-k1 selection fused into the epilogue so that the
 // B x N similarity matrix of Section 3.2's dense retrieval is never written out.
 //
-// Layout of one thread block (192 threads, one block per SM, persistent):
+// Layout of one thread block (224 threads, one block per SM, persistent):
 //   warp 0     TMA producer: streams 64-column slices of a bank tile (B operand, 256
-//              rows) into a shared-memory ring, 128-byte swizzled, K-major.  The query
-//              tile (A operand) is loaded once and stays in shared memory when the
-//              batch is small enough (<= 64 queries of width 1024); otherwise its
+//              rows) into a shared-memory ring of up to four stages, 128-byte swizzled,
+//              K-major (a last slice that reaches beyond the row width is zero-filled).
+//              The query tile (A operand) is loaded once and stays in shared memory when
+//              the batch is small enough (<= 64 queries of width 1024); otherwise its
 //              slices travel through the ring next to the bank's.  Small batches must
 //              not re-read the queries per bank tile: every block would ask L2 for
 //              the same few lines at the same moment.
-//   warp 1     MMA issuer: one thread issues tcgen05.mma 128x256x16 per 16 columns of
-//              a slice, accumulating D[query][bank row] in one of two 256-column
-//              tensor-memory buffers; tcgen05.commit hands smem stages back to the
-//              producer and finished accumulators to the epilogue.
-//   warps 2-5  epilogue: thread m owns query m of the tile (= TMEM lane m).  It reads
+//   warp 1     MMA issuer: one thread issues tcgen05.mma 128x256x16 (64x256x16 when at most
+//              64 queries are resident) per 16 columns of a slice, accumulating
+//              D[query][bank row] in one of two 256-column tensor-memory buffers;
+//              tcgen05.commit hands smem stages back to the producer and finished
+//              accumulators to the epilogue.
+//   warps 2-5  epilogue: a thread owns one query of the tile (its TMEM lane).  It reads
 //              its 256 similarities of a bank tile a chunk at a time, compares them with
 //              the query's running threshold held in a register, and appends the few
 //              survivors to the query's private candidate list in global memory.
 //              When a list fills, the warp cuts it back to its best k1 with an exact
 //              radix select over registers and the threshold rises.
-//   warp 6     threshold tracker: keeps re-reading the shared histograms of the block's
-//              128 queries and posts each query's current bin threshold in shared memory,
-//              so that the epilogue threads never wait on global memory between tiles.
+//   warp 6     threshold tracker (scans of two or more query tiles): re-reads the shared
+//              histograms of the block's queries on a thinning schedule and posts each
+//              query's current bin threshold in shared memory, so that the epilogue threads
+//              do not wait on global memory between tiles.
+//
+// With two or more query tiles, blocks run in clusters of two (cta_group::2): a pair shares
+// one 256-query x 256-row tile, each block loading its own queries and half of the bank slice.
 //
 // A bank tile is 256 consecutive entries; the queries sit on the accumulator's
 // lanes so that the per-query threshold test costs one register compare and no
@@ -33,17 +39,20 @@
 // the same time and share it through L2.
 //
 // The same kernel has a "dense" mode that writes every similarity of a small,
-// strided sample of the bank; its k1-th largest value per query is a safe starting
-// threshold for the full scan (at least k1 entries of the bank reach it).
+// strided sample of the bank; a value that at least k1 of a query's sampled similarities
+// reach is a safe starting threshold for the full scan (at least k1 entries of the bank
+// reach it).
 //
 // During the full scan the blocks tighten the thresholds together.  Each query has a
 // small histogram in global memory over the similarity range above its starting
-// threshold; every survivor is counted in it, the tracker warp reads the counters of the
-// block's queries over and over, and before each bank tile an epilogue thread raises its
-// threshold to the highest bin edge that was seen with k1 survivors at or above it.  Counters only grow, so whatever mix of old and new
-// values a reader sees undercounts, and a threshold derived from it still has at least
-// k1 real entries above it: the selection stays exact while the survivor rate falls
-// from k1/sample to about k1/(rows scanned so far by all blocks).
+// threshold; every survivor is counted in it, and a threshold is raised to the highest bin
+// edge that was seen with k1 survivors at or above it.  With one query tile the scan runs
+// at HBM speed and each epilogue thread reads its query's counters before every tile; with
+// more, the tensor cores set the pace, the thread reads them itself only for the first
+// tiles of a job and the tracker warp takes over.  Counters only grow, so whatever mix of
+// old and new values a reader sees undercounts, and a threshold derived from it still has
+// at least k1 real entries above it: the selection stays exact while the survivor rate
+// falls from k1/sample to about k1/(rows scanned so far by all blocks).
 //
 // Every wait on an mbarrier is bounded; a wait that runs out raises the block's
 // abort flag, every role leaves its loop, tensor memory is released and the status
