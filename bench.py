@@ -110,7 +110,8 @@ def time_oracle_sample(wl, bank_bits, q_tab, b, seconds, seed=0):
     """The CPU checker as it stands, on a bounded sample of the workload's queries."""
     import oracle
     from paper_2603_10846_b200 import synth
-    queries = synth.bf16_bits(synth.make_queries(wl, max(b, 1), "cpu", salt=99 + seed))
+    import torch
+    queries = synth.bf16_bits(synth.make_queries(wl, max(b, 1), "cpu", salt=99 + seed).to(dtype=torch.bfloat16))
     n_done, t0 = 0, time.perf_counter()
     ids_all = []
     while n_done < queries.shape[0]:
@@ -140,7 +141,7 @@ def run_reference(args):
     bank_bits = synth.bf16_bits(synth.make_bank(wl, "cpu").to(dtype=torch.bfloat16))
     q_tab = synth.make_q_tables(wl)
     total = args.steps + args.warmup
-    queries = synth.bf16_bits(synth.make_queries(wl, total + 1, "cpu", salt=7))
+    queries = synth.bf16_bits(synth.make_queries(wl, total + 1, "cpu", salt=7).to(dtype=torch.bfloat16))
     q = q_tab[0].copy()
 
     def step(i, rows):
