@@ -391,7 +391,10 @@ def run_evk(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{wl.name}: N={wl.n}, d={wl.d} bf16, B={b}, k1={wl.k1}, k2={wl.k2}, w={wl.w}; "
                                    f"step = insert {n_new} + retrieve {b} + update {n_upd * world}",
-                       "l2": "inputs larger than L2 (bank %.2f GiB scanned every step)" % (size * wl.d * 2 / 2 ** 30),
+                       "l2": ("inputs larger than L2 (bank %.2f GiB scanned every step)" % (size * wl.d * 2 / 2 ** 30))
+                       if size * wl.d * 2 > 126e6 else
+                       "bank of %.1f MiB fits in L2 and is not flushed between steps: a parity workload, not a bench line"
+                       % (size * wl.d * 2 / 2 ** 20),
                        "parallelism": "replicated bank, queries sharded by rank, update batches all-gathered"
                        if world > 1 else "single GPU"},
             "entries_scanned_per_s": value * size,
