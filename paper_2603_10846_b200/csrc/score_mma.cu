@@ -152,6 +152,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// The same load with an L2 eviction-priority hint (see l2_evict_first_policy).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+// "Evict this first": for data that is read once, so that it does not push out lines that are
+// read again and again (the queries, the histograms, the candidate lists).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
@@ -451,6 +467,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = !(p.stall && p.mode == 0);
+            // one query tile: every bank tile is read by exactly one block, once
+            const bool stream_once = !kPair && p.n_qt == 1 && p.mode == 0;
+            const uint64_t bank_policy = l2_evict_first_policy();
             if (ok && p.a_resident && worker < n_jobs) {
                 mbar_arrive_expect_tx(afull, a_region);
                 for (int kc = 0; kc < k_chunks; ++kc) tma_load_2d(tiles + kc * a_slice, &map_q, afull, kc * kBlockK, 0);
@@ -472,7 +491,10 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         } else {
                             mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
                             if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
-                            tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
+                            if (stream_once)
+                                tma_load_2d_hint(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN, bank_policy);
+                            else
+                                tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
