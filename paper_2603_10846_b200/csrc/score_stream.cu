@@ -24,12 +24,19 @@ constexpr int kRowsPerIter = kWarps * kRowsPerWarp;  // rows a block takes per i
 constexpr int kSelPerThread = 8;                     // capacity <= kThreads * kSelPerThread
 constexpr int kMaxCap = kThreads * kSelPerThread;    // 2048
 
-__device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
+// A bank row is read once per launch: no L1 allocation, and first in line for eviction from L2 so
+// that the stream does not push out what is read again (queries, candidate lists).
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p, uint64_t policy) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
+                 : "l"(p), "l"(policy));
     return v;
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
 }
 
 // QB queries per pass, NCH 16-byte chunks of a row per lane (row width d <= NCH*256).
@@ -75,6 +82,7 @@ score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
     }
     __syncthreads();
 
+    const uint64_t policy = l2_evict_first_policy();
     const int64_t n_iters = (size + kRowsPerIter - 1) / kRowsPerIter;
     for (int64_t it = blockIdx.x; it < n_iters; it += gridDim.x) {
         const int64_t row0 = it * kRowsPerIter + warp * kRowsPerWarp;
@@ -88,7 +96,7 @@ score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
 #pragma unroll
                 for (int j = 0; j < NCH; ++j) {
                     const int c = lane + 32 * j;
-                    v[r][j] = (row < size && c < chunks) ? ldg_stream(src + c) : make_uint4(0, 0, 0, 0);
+                    v[r][j] = (row < size && c < chunks) ? ldg_stream(src + c, policy) : make_uint4(0, 0, 0, 0);
                 }
             }
             float acc[2][QB];
