@@ -10,6 +10,7 @@ namespace {
 constexpr int kThreads = 256;
 
 // 8 elements per thread: two 16-byte loads of fp32 (or one of bf16), one 16-byte store.
+// (the query conversion; inserts use insert_kernel below)
 __global__ void __launch_bounds__(kThreads)
 insert_rows_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int is_bf16, int64_t n_vec) {
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * kThreads) {
@@ -32,10 +33,30 @@ insert_rows_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src
     }
 }
 
+// Rows and values of an insert in one launch (an insert of a few rows is all launch latency).
 __global__ void __launch_bounds__(kThreads)
-insert_values_kernel(float *__restrict__ q_tables, uint32_t *__restrict__ visits, int64_t capacity, int n_stages,
-                     int64_t first, int64_t n,
-                     int stage, const float *__restrict__ q_init, float q_default, int32_t *__restrict__ ids_out) {
+insert_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int is_bf16, int64_t n_vec,
+              float *__restrict__ q_tables, uint32_t *__restrict__ visits, int64_t capacity, int n_stages,
+              int64_t first, int64_t n, int stage, const float *__restrict__ q_init, float q_default,
+              int32_t *__restrict__ ids_out) {
+    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * kThreads) {
+        uint4 out;
+        if (is_bf16) {
+            out = reinterpret_cast<const uint4 *>(src)[i];
+        } else {
+            const float4 a = reinterpret_cast<const float4 *>(src)[2 * i];
+            const float4 b = reinterpret_cast<const float4 *>(src)[2 * i + 1];
+            __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y);
+            __nv_bfloat162 p1 = __floats2bfloat162_rn(a.z, a.w);
+            __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y);
+            __nv_bfloat162 p3 = __floats2bfloat162_rn(b.z, b.w);
+            out.x = *reinterpret_cast<uint32_t *>(&p0);
+            out.y = *reinterpret_cast<uint32_t *>(&p1);
+            out.z = *reinterpret_cast<uint32_t *>(&p2);
+            out.w = *reinterpret_cast<uint32_t *>(&p3);
+        }
+        reinterpret_cast<uint4 *>(dst)[i] = out;
+    }
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kThreads) {
         const float v = q_init ? q_init[i] : q_default;
         for (int s = 0; s < n_stages; ++s) {
@@ -62,11 +83,9 @@ cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits
                           cudaStream_t stream, int *launches) {
     if (n <= 0) return cudaSuccess;
     const int64_t n_vec = n * d / 8;
-    insert_rows_kernel<<<grid_for(n_vec), kThreads, 0, stream>>>(bank + first * d, emb, emb_dtype == EVK_DTYPE_BF16, n_vec);
-    ++*launches;
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
-    insert_values_kernel<<<grid_for(n), kThreads, 0, stream>>>(q_tables, visits, capacity, n_stages, first, n, stage, q_init, q_default, ids_out);
+    insert_kernel<<<grid_for(n_vec > n ? n_vec : n), kThreads, 0, stream>>>(
+        bank + first * d, emb, emb_dtype == EVK_DTYPE_BF16, n_vec, q_tables, visits, capacity, n_stages, first, n,
+        stage, q_init, q_default, ids_out);
     ++*launches;
     return cudaGetLastError();
 }
