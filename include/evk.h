@@ -180,7 +180,10 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
  *     library, for the life of the process, whether or not this call is used.
  *   - The first call on each device looks up the array's device address (with that
  *     device current, which it must be at every call); make that first call before
- *     any stream capture begins.  The call itself allocates and frees nothing.
+ *     any stream capture begins.  The call itself allocates and frees nothing.  The address is
+ *     remembered per device ordinal (ordinals 0..63; a higher one returns EVK_ERR_CUDA) for the
+ *     life of the process: after cudaDeviceReset, or anything else that destroys the device's
+ *     primary context, it is stale and this call must not be used again in that process.
  *   - Every call on a device shares the one array.  Calls are safe one after
  *     another on one stream; two calls whose kernels can overlap on the GPU
  *     (different streams without ordering) race on the scratch and corrupt each

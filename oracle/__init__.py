@@ -52,6 +52,8 @@ def _load():
     lib.evk_oracle_threads.restype = ctypes.c_int
     lib.evk_oracle_sims.argtypes = [p, c_i64, c_i32, p, p]
     lib.evk_oracle_sims.restype = None
+    lib.evk_oracle_rank.argtypes = [p, c_i64, c_i32, p, p]
+    lib.evk_oracle_rank.restype = c_i32
     lib.evk_oracle_phase1.argtypes = [p, c_i64, c_i32, p, c_i32, p, p]
     lib.evk_oracle_phase1.restype = c_i32
     lib.evk_oracle_phase2.argtypes = [p, p, c_i32, p, c_f64, c_i32, p, p]
@@ -121,6 +123,17 @@ def sims(bank_bits, query_bits) -> np.ndarray:
     out = np.empty(size, dtype=np.float64)
     _load().evk_oracle_sims(_ptr(bank_bits), size, d, _ptr(query_bits), _ptr(out))
     return out
+
+
+def rank(sims_row, k1: int):
+    """The ranking step of phase 1 on one query's similarities (entry id = index): the first k1
+    by (similarity desc, id asc) after a full sort.  ids int32 [k1], sims fp64 [k1]."""
+    sims_row = _c(sims_row, np.float64)
+    assert sims_row.ndim == 1
+    ids = np.empty(k1, dtype=np.int32)
+    sm = np.empty(k1, dtype=np.float64)
+    _load().evk_oracle_rank(_ptr(sims_row), sims_row.size, k1, _ptr(ids), _ptr(sm))
+    return ids, sm
 
 
 def phase1(bank_bits, query_bits, k1: int):

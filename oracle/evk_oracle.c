@@ -98,22 +98,31 @@ static int ranked_cmp(const void *a, const void *b) {
     return (x->id > y->id) - (x->id < y->id);
 }
 
-/* The top-K candidate pool C(x): all `size` similarities, fully sorted by
- * (similarity descending, id ascending); the first min(k1, size) are the pool.
- * Unused slots get id -1 and similarity -inf.  Returns the pool length. */
-int32_t evk_oracle_phase1(const uint16_t *bank, int64_t size, int32_t d,
-                          const uint16_t *query, int32_t k1,
-                          int32_t *pool_ids, double *pool_sims) {
+/* Ranking step of the candidate pool: the `size` similarities sims[] (entry id = index) are
+ * fully sorted by (similarity descending, id ascending); the first min(k1, size) are the
+ * pool.  Unused slots get id -1 and similarity -inf.  Returns the pool length. */
+int32_t evk_oracle_rank(const double *sims, int64_t size, int32_t k1,
+                        int32_t *pool_ids, double *pool_sims) {
     int32_t n_pool = (int32_t)((int64_t)k1 < size ? (int64_t)k1 : size);
     for (int32_t j = 0; j < k1; ++j) { pool_ids[j] = -1; pool_sims[j] = -INFINITY; }
     if (size <= 0) return 0;
-    double *sims = (double *)malloc((size_t)size * sizeof(double));
     ranked_t *r = (ranked_t *)malloc((size_t)size * sizeof(ranked_t));
-    evk_oracle_sims(bank, size, d, query, sims);
     for (int64_t i = 0; i < size; ++i) { r[i].key = sims[i]; r[i].key2 = 0.0; r[i].id = (int32_t)i; }
     qsort(r, (size_t)size, sizeof(ranked_t), ranked_cmp);
     for (int32_t j = 0; j < n_pool; ++j) { pool_ids[j] = r[j].id; pool_sims[j] = r[j].key; }
     free(r);
+    return n_pool;
+}
+
+/* The top-K candidate pool C(x): every stored entry's similarity (evk_oracle_sims), then the
+ * ranking step above. */
+int32_t evk_oracle_phase1(const uint16_t *bank, int64_t size, int32_t d,
+                          const uint16_t *query, int32_t k1,
+                          int32_t *pool_ids, double *pool_sims) {
+    if (size <= 0) return evk_oracle_rank(NULL, 0, k1, pool_ids, pool_sims);
+    double *sims = (double *)malloc((size_t)size * sizeof(double));
+    evk_oracle_sims(bank, size, d, query, sims);
+    const int32_t n_pool = evk_oracle_rank(sims, size, k1, pool_ids, pool_sims);
     free(sims);
     return n_pool;
 }

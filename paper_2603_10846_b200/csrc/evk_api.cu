@@ -1,5 +1,6 @@
 // The C ABI (include/evk.h): argument checks, memory layout, kernel dispatch.
 #include <math.h>
+#include <mutex>
 #include <new>
 #include <string.h>
 
@@ -7,6 +8,26 @@
 #include "evk_kernels.cuh"
 
 using namespace evk;
+
+namespace evk {
+int num_sms() {
+    constexpr int kFallback = 148, kMaxDev = 64;
+    static std::mutex mu;
+    static int cache[kMaxDev];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) {
+        (void)cudaGetLastError();
+        return kFallback;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 2) n = kFallback;
+        cache[dev] = n;
+    }
+    return cache[dev];
+}
+}  // namespace evk
 
 struct evk_mem {
     evk_config cfg;
@@ -387,11 +408,16 @@ int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32
                       int32_t k1, int32_t k2, float w,
                       int32_t *ids_out_host, float *scores_out_host,
                       void *workspace, size_t workspace_bytes, void *stream_v) {
-    if (!mem || B < 0 || k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return EVK_ERR_INVALID;
+    // every check evk_retrieve makes on the host is made here first: nothing is copied for a call
+    // that would be refused
+    if (!mem || B < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (k1 < 1 || k1 > EVK_MAX_K1 || k2 < 1 || k2 > k1) return EVK_ERR_INVALID;
+    if (!(w >= 0.0f && w <= 1.0f)) return EVK_ERR_INVALID;
     if (q_dtype != EVK_DTYPE_F32 && q_dtype != EVK_DTYPE_BF16) return EVK_ERR_INVALID;
     if (B == 0) return EVK_OK;
     if (!queries_host || !ids_out_host || !scores_out_host || !workspace || !aligned(workspace, 256))
         return EVK_ERR_INVALID;
+    if (pick_kind(mem, B, k1) == 0) return EVK_ERR_UNSUPPORTED;
     if (workspace_bytes < evk_retrieve_host_workspace_bytes(mem, B, k1, k2)) return EVK_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const size_t b = (size_t)B;
@@ -404,13 +430,17 @@ int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32
     const size_t inner_bytes = workspace_bytes - (size_t)(inner - ws);
     if (cudaMemcpyAsync(q_dev, queries_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return EVK_ERR_CUDA;
+    // from here on a copy may be in flight: every return synchronises, so that the caller's host
+    // buffers are its own again whatever the outcome
     int rc = evk_retrieve(mem, q_dev, q_dtype, B, stage, k1, k2, w, ids_dev, scores_dev, nullptr, nullptr,
                           inner, inner_bytes, stream_v);
-    if (rc != EVK_OK) return rc;
-    if (cudaMemcpyAsync(ids_out_host, ids_dev, b * k2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaMemcpyAsync(scores_out_host, scores_dev, b * k2 * sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-        return EVK_ERR_CUDA;
-    return cuda_status(cudaStreamSynchronize(stream));
+    if (rc == EVK_OK &&
+        (cudaMemcpyAsync(ids_out_host, ids_dev, b * k2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+         cudaMemcpyAsync(scores_out_host, scores_dev, b * k2 * sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess))
+        rc = EVK_ERR_CUDA;
+    const cudaError_t sync = cudaStreamSynchronize(stream);
+    if (rc == EVK_OK && sync != cudaSuccess) rc = EVK_ERR_CUDA;
+    return rc;
 }
 
 size_t evk_q_update_host_workspace_bytes(const evk_mem *mem, int64_t M) {
@@ -421,8 +451,11 @@ size_t evk_q_update_host_workspace_bytes(const evk_mem *mem, int64_t M) {
 int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stage,
                       const float *rewards_host, float alpha,
                       void *workspace, size_t workspace_bytes, void *stream_v) {
-    if (!mem || M < 0) return EVK_ERR_INVALID;
+    // the host-side checks of evk_q_update, before anything is copied
+    if (!mem || M < 0 || !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (!(alpha > 0.0f && alpha <= 1.0f)) return EVK_ERR_INVALID;
     if (M == 0) return EVK_OK;
+    if (M >= ((int64_t)1 << 31)) return EVK_ERR_UNSUPPORTED;
     if (!ids_host || !rewards_host || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
     if (workspace_bytes < evk_q_update_host_workspace_bytes(mem, M)) return EVK_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -430,12 +463,17 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
     int32_t *ids_dev = reinterpret_cast<int32_t *>(ws);
     float *r_dev = reinterpret_cast<float *>(ws + align256((size_t)M * 4));
     char *inner = ws + 2 * align256((size_t)M * 4);
-    if (cudaMemcpyAsync(ids_dev, ids_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-        cudaMemcpyAsync(r_dev, rewards_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    int rc = EVK_OK;
+    if (cudaMemcpyAsync(ids_dev, ids_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return EVK_ERR_CUDA;
-    int rc = evk_q_update(mem, ids_dev, M, stage, r_dev, alpha, inner, workspace_bytes - (size_t)(inner - ws), stream_v);
-    if (rc != EVK_OK) return rc;
-    return cuda_status(cudaStreamSynchronize(stream));
+    // a copy may be in flight from here on: every return synchronises first
+    if (cudaMemcpyAsync(r_dev, rewards_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        rc = EVK_ERR_CUDA;
+    if (rc == EVK_OK)
+        rc = evk_q_update(mem, ids_dev, M, stage, r_dev, alpha, inner, workspace_bytes - (size_t)(inner - ws), stream_v);
+    const cudaError_t sync = cudaStreamSynchronize(stream);
+    if (rc == EVK_OK && sync != cudaSuccess) rc = EVK_ERR_CUDA;
+    return rc;
 }
 
 // ---- exploration -----------------------------------------------------------------

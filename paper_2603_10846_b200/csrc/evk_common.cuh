@@ -9,7 +9,11 @@
 
 namespace evk {
 
-constexpr int kNumSM = 148;            // B200: 2 dies x 74 SMs
+// Streaming multiprocessors of the current device (cudaDevAttrMultiProcessorCount, asked once per
+// device; 148 on a B200: 2 dies x 74).  Grids, bank splits and workspace sizes follow it, so a
+// workspace must be sized and used with the same device current.  Falls back to 148 when no
+// device can be asked (sizes queried on a machine without a GPU).
+int num_sms();
 constexpr uint32_t kPadId = 0xffffffffu;
 
 // ---------------------------------------------------------------------------

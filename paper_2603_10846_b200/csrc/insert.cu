@@ -69,7 +69,7 @@ insert_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int
 
 int grid_for(int64_t work_items) {
     int64_t g = (work_items + kThreads - 1) / kThreads;
-    const int64_t cap = (int64_t)kNumSM * 8;
+    const int64_t cap = (int64_t)num_sms() * 8;
     if (g > cap) g = cap;
     if (g < 1) g = 1;
     return (int)g;

@@ -317,7 +317,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
     cudaError_t err = cudaMemsetAsync(flags, 0, sizeof(int), stream);
     if (err != cudaSuccess) return err;
     int vgrid = (int)((m + kThreads - 1) / kThreads);
-    if (vgrid > kNumSM * 8) vgrid = kNumSM * 8;
+    if (vgrid > num_sms() * 8) vgrid = num_sms() * 8;
     validate_kernel<<<vgrid, kThreads, 0, stream>>>(ids, rewards, m, size, flags);
     ++*launches;
 

@@ -90,7 +90,7 @@ reward_normalize_kernel(double *__restrict__ state, const float *__restrict__ ra
 
 int grid_for(int64_t n) {
     int64_t g = (n + kThreads - 1) / kThreads;
-    if (g > kNumSM * 8) g = kNumSM * 8;
+    if (g > num_sms() * 8) g = num_sms() * 8;
     return (int)(g < 1 ? 1 : g);
 }
 

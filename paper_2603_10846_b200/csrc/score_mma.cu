@@ -55,8 +55,9 @@
 // falls from k1/sample to about k1/(rows scanned so far by all blocks).
 //
 // Every wait on an mbarrier is bounded; a wait that runs out raises the block's
-// abort flag, every role leaves its loop, tensor memory is released and the status
-// word reports EVK_ERR_DEVICE_TIMEOUT.
+// abort flag, every role leaves its loop, the producer waits (bounded again) for the
+// copies it still has in flight, tensor memory is released and the status word
+// reports EVK_ERR_DEVICE_TIMEOUT.
 #include <cuda.h>
 
 #include "evk_common.cuh"
@@ -145,6 +146,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return true;
 }
 
+// Bounded wait that ignores the abort flag (used once the block is already backing out).
+__device__ __forceinline__ bool mbar_wait_deadline(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > limit) return false;
+    }
+    return true;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -218,6 +228,9 @@ __device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -423,6 +436,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // (query << 32 | bin threshold) coming back; epi_done counts epilogue warps that have finished
     volatile int *epi_done = reinterpret_cast<volatile int *>(tmem_slot + 2);
     volatile int *tile_seq = reinterpret_cast<volatile int *>(tmem_slot + 3);   // accumulators examined so far
+    // written by the partner block of a pair at teardown: slices its producer issued, its abort flag
+    volatile int *peer_issued = reinterpret_cast<volatile int *>(tmem_slot + 4);
+    volatile int *peer_abort = reinterpret_cast<volatile int *>(tmem_slot + 5);
     volatile int *slot_q = reinterpret_cast<volatile int *>(reinterpret_cast<unsigned char *>(bars) + 256);
     volatile unsigned long long *slot_tau =
         reinterpret_cast<volatile unsigned long long *>(reinterpret_cast<unsigned char *>(bars) + 256 + 512);
@@ -468,6 +484,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (kPair) cluster_sync_all();  // the partner's barriers exist before anything is signalled across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // the producer's record of what it has put in flight (thread 0 only), for the teardown
+    int n_issued = 0;        // ring slices armed and issued so far
+    bool a_armed = false;    // the resident query tile was requested
 
     if (warp == 0) {
         // ===== TMA producer =====
@@ -480,6 +499,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const bool stream_once = p.mode == 0 && (kPair ? p.n_qt <= 2 : p.n_qt == 1);
             const uint64_t bank_policy = l2_evict_first_policy();
             if (ok && p.a_resident && worker < n_jobs) {
+                a_armed = true;
                 mbar_arrive_expect_tx(afull, a_region);
                 for (int kc = 0; kc < k_chunks; ++kc) tma_load_2d(tiles + kc * a_slice, &map_q, afull, kc * kBlockK, 0);
             }
@@ -509,6 +529,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                             else
                                 tma_load_2d(s_dst + b_off, &map_bank, full0 + 8 * stage, kc * kBlockK, t * kBlockN);
                         }
+                        ++n_issued;
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                 }
@@ -781,10 +802,48 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // ===== teardown =====
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
-        // give copies still in flight time to land before shared memory is released
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)EVK_ERR_DEVICE_TIMEOUT);
+    const int aborted = *abort_flag;
+    if (kPair) {
+        // each block tells its partner how far its producer got and whether it is backing out
+        if (threadIdx.x == 0) {
+            st_cluster_u32(mapa_u32(smem_u32(const_cast<int *>(peer_issued)), rank ^ 1u), (uint32_t)n_issued);
+            st_cluster_u32(mapa_u32(smem_u32(const_cast<int *>(peer_abort)), rank ^ 1u), (uint32_t)aborted);
+        }
+        cluster_sync_all();
+    }
+    if (aborted || (kPair && *peer_abort)) {
+        // Backing out: no copy may still be on its way into this block's shared memory when the block
+        // ends.  Both producers have left their loops, so nothing new is issued except the stand-ins
+        // below; then the thread that armed the full barriers waits, bounded, for every phase it or
+        // its partner counted bytes on.
+        if (threadIdx.x == 0) {
+            int n_all = n_issued;
+            if (kPair) {
+                // The two producers of a pair are never more than a ring apart (a slice is issued only
+                // after the MMA that consumed the slice one ring earlier, which needed both halves).
+                // The one that stopped first issues stand-in loads (tile 0) for the slices its partner
+                // still issued, so that every such phase of the leader's barriers completes.
+                const int n_peer = *peer_issued;
+                for (int i = n_issued; i < n_peer; ++i) {
+                    const int s = i % kStages;
+                    const uint32_t s_dst = ring + s * stage_bytes;
+                    const uint32_t leader_full = mapa_u32(full0 + 8 * s, 0);
+                    if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * s, 2 * stage_bytes);
+                    tma_load_2d_pair(s_dst, &map_q, leader_full, 0, 0);
+                    tma_load_2d_pair(s_dst + b_off, &map_bank, leader_full, 0, 0);
+                }
+                if (n_peer > n_all) n_all = n_peer;
+            }
+            if (rank == 0) {   // the bytes of both blocks of a pair are counted on the leader's barriers
+                if (a_armed) mbar_wait_deadline(afull, 0, wait_limit);
+                for (int s = 0; s < kStages; ++s) {
+                    if (n_all <= s) break;
+                    const int last = s + kStages * ((n_all - 1 - s) / kStages);   // last slice that used stage s
+                    mbar_wait_deadline(full0 + 8 * s, (uint32_t)(last / kStages) & 1u, wait_limit);
+                }
+            }
+            if (aborted) atomicCAS(p.status, 0, (int)EVK_ERR_DEVICE_TIMEOUT);
+        }
         __syncthreads();
     }
     if (kPair) cluster_sync_all();  // neither block frees tensor memory or leaves while the other may touch it
@@ -1011,7 +1070,7 @@ bool use_pairs(int n_qt) { return n_qt >= 2; }
 int splits_for(int n_qt, int n_tiles) {
     if (n_qt <= 0) n_qt = 1;
     // workers: single blocks, or pairs of blocks that take two query tiles at a time
-    const int n_work = use_pairs(n_qt) ? kNumSM / 2 : kNumSM;
+    const int n_work = use_pairs(n_qt) ? num_sms() / 2 : num_sms();
     const int n_units = use_pairs(n_qt) ? (n_qt + 1) / 2 : n_qt;
     int base = n_work / n_units;
     if (base < 1) base = 1;
@@ -1065,10 +1124,10 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     pl.pair = use_pairs(pl.n_qt) ? 1 : 0;
     if (pl.pair) {
         const int jobs = ((pl.n_qt + 1) / 2) * pl.splits;
-        pl.grid = 2 * (jobs < kNumSM / 2 ? jobs : kNumSM / 2);
+        pl.grid = 2 * (jobs < num_sms() / 2 ? jobs : num_sms() / 2);
     } else {
         const int jobs = pl.n_qt * pl.splits;
-        pl.grid = jobs < kNumSM ? jobs : kNumSM;
+        pl.grid = jobs < num_sms() ? jobs : num_sms();
     }
     if (pl.grid < 1) pl.grid = 1;
     // a strided sample of the bank gives each query a starting threshold
@@ -1133,12 +1192,12 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.mode = 1;
         p.n_tiles = pl.n_sample / kBlockN;
         // the sample pass is small: single blocks, as many splits as fit next to the query tiles
-        int s_splits = kNumSM / p.n_qt;
+        int s_splits = num_sms() / p.n_qt;
         if (s_splits < 1) s_splits = 1;
         if (s_splits > p.n_tiles) s_splits = p.n_tiles;
         p.splits = s_splits;
         const int jobs = p.n_qt * p.splits;
-        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < kNumSM ? jobs : kNumSM, sp.bytes, false, false, stream);
+        cudaError_t err = launch_kernel(map_q, map_sample, p, jobs < num_sms() ? jobs : num_sms(), sp.bytes, false, false, stream);
         if (err != cudaSuccess) return err;
         ++*launches;
         {

@@ -266,7 +266,7 @@ StreamPlan stream_plan(int64_t size, int d, int B, int k1) {
     int ctas_per_sm = blocks_per_sm_for(p.qb, nch, p.smem);
     if (ctas_per_sm > 4) ctas_per_sm = 4;
     int64_t iters = (size + kRowsPerIter - 1) / kRowsPerIter;
-    int64_t grid = (int64_t)kNumSM * ctas_per_sm;
+    int64_t grid = (int64_t)num_sms() * ctas_per_sm;
     if (grid > iters) grid = iters;
     if (grid < 1) grid = 1;
     p.nparts = (int)grid;

@@ -120,7 +120,7 @@ cudaError_t launch_tag_pool(const int32_t *pool_ids, int64_t n, int32_t id_offse
                             int32_t *gids_out, float *q_out, cudaStream_t stream, int *launches) {
     if (n <= 0) return cudaSuccess;
     int64_t grid = (n + kTagThreads - 1) / kTagThreads;
-    if (grid > kNumSM * 8) grid = kNumSM * 8;
+    if (grid > num_sms() * 8) grid = num_sms() * 8;
     ++*launches;
     return launch_overlapped(tag_pool_kernel, dim3((unsigned)grid), dim3(kTagThreads), 0, stream, pool_ids, n,
                              id_offset, q_stage, gids_out, q_out);

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Exact-match rates of the parity cases against the oracle (the band rule accepts a swap at a
+    pool or result boundary within tolerance; this says how often one happened)."""
+    from tests import parity
+    if parity.REPORT:
+        terminalreporter.write_sep("-", "parity: share of judged queries whose id sets equal the oracle's")
+        for line in parity.REPORT:
+            terminalreporter.write_line(line)

@@ -20,19 +20,28 @@ import oracle
 REL = 2e-3
 ABS = 1e-5
 
+# Realised exact-match rates, one line per judged case; printed at the end of the test run.
+REPORT = []
+
+
+def record(case, scoring, judged, batch, exact_pool, exact_final):
+    kind = {None: "auto", 1: "stream", 2: "tensor"}.get(scoring, str(scoring))
+    REPORT.append(f"{case:44s} kernel={kind:6s} judged {judged:4d} of {batch:4d}: "
+                  f"pool ids exact {100 * exact_pool:6.2f} %, result ids exact {100 * exact_final:6.2f} %")
+
 
 def tol(score, scale=1.0):
     return REL * np.abs(score) + ABS * scale
 
 
-def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0):
-    """Phase 1 of one query.  Returns True if the id set equals the oracle's exactly."""
+def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0, sims=None):
+    """Phase 1 of one query.  Returns True if the id set equals the oracle's exactly.
+    sims: this query's oracle similarities if the caller already has them."""
     size = bank_bits.shape[0]
     n_pool = min(k1, size)
-    sims = oracle.sims(bank_bits, query_bits) if size else np.zeros(0)
-    o_ids, o_sims = oracle.phase1(bank_bits, query_bits, k1) if size else (
-        np.full((1, k1), -1, np.int32), np.full((1, k1), -np.inf))
-    o_ids, o_sims = o_ids[0], o_sims[0]
+    if sims is None:
+        sims = oracle.sims(bank_bits, query_bits) if size else np.zeros(0)
+    o_ids, o_sims = oracle.rank(sims, k1)
     pool_ids = np.asarray(pool_ids)
     pool_sims = np.asarray(pool_sims, dtype=np.float64)
     # shape of the answer: n_pool real entries, then padding
@@ -58,7 +67,8 @@ def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0):
     return set(real.tolist()) == set(o_ids[:n_pool].tolist())
 
 
-def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, norm_scale=1.0, zscore=False):
+def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, norm_scale=1.0, zscore=False,
+                sims=None):
     """Phase 2 of one query, judged on the library's own pool.  zscore: the pool z-score variant."""
     pool_ids = np.asarray(pool_ids)
     ids = np.asarray(ids)
@@ -68,7 +78,8 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
     assert np.all(ids[n_out:] == -1) and np.all(np.isneginf(scores[n_out:])), "bad padding"
     if n_out == 0:
         return True
-    sims = oracle.sims(bank_bits, query_bits)
+    if sims is None:
+        sims = oracle.sims(bank_bits, query_bits)
     o_ids, o_sc = oracle.phase2(real, sims[real], q_stage, w, real.size, zscore)   # the whole pool, ranked
     o_ids, o_sc = o_ids[0], o_sc[0]
     score_of = dict(zip(o_ids.tolist(), o_sc.tolist()))
@@ -92,19 +103,32 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
     return got.tolist() == o_ids[:n_out].tolist()
 
 
-def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None, norm_scale=1.0, zscore=False):
-    """out = (ids, scores, pool_ids, pool_sims) as host arrays; sample = query indices to judge."""
+def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None, norm_scale=1.0, zscore=False,
+                   workers=4):
+    """out = (ids, scores, pool_ids, pool_sims) as host arrays; sample = query indices to judge.
+    Returns the share of judged queries whose pool, and whose result, equal the oracle's exactly.
+    Each judged query costs the oracle one scan of the bank and one full sort; `workers` queries are
+    judged side by side (threads: the oracle's C calls release the interpreter lock)."""
     ids, scores, pool_ids, pool_sims = [np.asarray(x) for x in out]
     b = queries_bits.shape[0]
-    sample = range(b) if sample is None else sample
-    exact_pool = exact_final = 0
-    n = 0
-    for i in sample:
-        exact_pool += bool(check_pool(bank_bits, queries_bits[i], k1, pool_ids[i], pool_sims[i], norm_scale))
-        exact_final += bool(check_final(bank_bits, queries_bits[i], q_stage, w, k2, pool_ids[i], ids[i],
-                                        scores[i], norm_scale, zscore))
-        n += 1
-    return exact_pool / max(n, 1), exact_final / max(n, 1)
+    sample = list(range(b) if sample is None else sample)
+    size = bank_bits.shape[0]
+
+    def judge(i):
+        sims = oracle.sims(bank_bits, queries_bits[i]) if size else np.zeros(0)
+        ep = bool(check_pool(bank_bits, queries_bits[i], k1, pool_ids[i], pool_sims[i], norm_scale, sims=sims))
+        ef = bool(check_final(bank_bits, queries_bits[i], q_stage, w, k2, pool_ids[i], ids[i], scores[i],
+                              norm_scale, zscore, sims=sims))
+        return ep, ef
+
+    if workers > 1 and len(sample) > 1 and size * bank_bits.shape[1] > (1 << 22):
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(workers) as pool:
+            res = list(pool.map(judge, sample))
+    else:
+        res = [judge(i) for i in sample]
+    n = max(len(res), 1)
+    return sum(r[0] for r in res) / n, sum(r[1] for r in res) / n
 
 
 def check_update(q_before, ids, rewards, alpha, q_after):

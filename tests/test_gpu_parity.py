@@ -88,7 +88,21 @@ def test_tiny_fp32_bank_both_stages_then_updates(evk):
     parity.check_retrieve(bank_bits, q_bits, q_after, wl.k1, wl.k2, wl.w, out)
 
 
-def _workload_case(evk, name, b, n_oracle, stage=0, scoring=None, n=None):
+def tile_sample(b, per_tile, seed=0, tile=128):
+    """Query indices that hit every 128-query tile of the batch (so both blocks of every pair of
+    tiles): per tile its first and last row, then random rows, `per_tile` in all."""
+    rng = np.random.default_rng(seed)
+    picked = []
+    for t0 in range(0, b, tile):
+        rows = np.arange(t0, min(b, t0 + tile))
+        must = [rows[0], rows[-1]][:per_tile]
+        rest = np.setdiff1d(rows, must)
+        extra = rng.choice(rest, min(max(per_tile - len(must), 0), rest.size), replace=False)
+        picked += sorted(set(int(x) for x in must) | set(int(x) for x in extra))
+    return picked
+
+
+def _workload_case(evk, name, b, sample, stage=0, scoring=None, n=None, label=None):
     wl = synth.WORKLOADS[name]
     bank = synth.make_bank(wl, DEV, n=n)
     queries = synth.make_queries(wl, b, DEV)
@@ -96,39 +110,99 @@ def _workload_case(evk, name, b, n_oracle, stage=0, scoring=None, n=None):
     mem = make_mem(evk, bank, q_tab, scoring=scoring)
     out = run_retrieve(evk, mem, queries, stage, wl.k1, wl.k2, wl.w)
     bank_bits, q_bits = host_bits(bank), host_bits(queries)
-    ep, ef = parity.check_retrieve(bank_bits, q_bits, q_tab[stage], wl.k1, wl.k2, wl.w, out,
-                                   sample=sample_of(b, n_oracle))
+    ep, ef = parity.check_retrieve(bank_bits, q_bits, q_tab[stage], wl.k1, wl.k2, wl.w, out, sample=sample)
+    n_judged = b if sample is None else len(sample)
+    parity.record(label or f"{name} B={b}", scoring, n_judged, b, ep, ef)
     assert ep >= 0.9 and ef >= 0.9
     return wl, mem, q_tab
 
 
 def test_mid_bank_retrieve_and_lognormal_updates(evk, scoring):
-    wl, mem, q_tab = _workload_case(evk, "mid", 256, 24, stage=1, scoring=scoring)
+    # every one of the 256 queries is judged
+    wl, mem, q_tab = _workload_case(evk, "mid", 256, None, stage=1, scoring=scoring)
     ids, r = synth.make_updates(wl)
     evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 1, torch.from_numpy(r).to(DEV), wl.alpha)
     parity.check_update(q_tab[1], ids, r, wl.alpha, evk.evk_q_read(mem, 1).cpu().numpy())
 
 
 def test_clustered_bank(evk, scoring):
-    _workload_case(evk, "clustered", 1024, 12, scoring=scoring)
+    # 128 of the 1,024 queries: 16 in each of the 8 query tiles
+    _workload_case(evk, "clustered", 1024, tile_sample(1024, 16, seed=2), scoring=scoring)
 
 
 @pytest.mark.parametrize("b", [1, 8, 64])
 def test_large_bank_small_batches(evk, b, scoring):
-    _workload_case(evk, "large_hbm", b, 6, scoring=scoring)
+    _workload_case(evk, "large_hbm", b, None, scoring=scoring)     # every query is judged
 
 
-def test_large_bank_big_batch_with_zipf_updates(evk, scoring):
-    wl, mem, q_tab = _workload_case(evk, "large_compute", 4096, 4, scoring=scoring)
-    q = q_tab.copy()
-    for rnd in range(3):                       # streaming updates, stage alternating by round
+def test_large_bank_interleaved_retrievals_and_zipf_updates(evk, scoring):
+    """The streaming protocol as configured: rounds of retrieve (4,096 fresh queries) -> update
+    (65,536 popularity-skewed ids), the stage alternating by round.  From round 2 on a retrieval
+    reads a value table that an earlier round's update wrote (Section 3.2's phase 2 fed by Eq. 4).
+    The oracle keeps its own tables, advanced by its own binary32 update; nothing the library
+    returns ever goes into them."""
+    wl = synth.WORKLOADS["large_compute"]
+    b = max(wl.batches)
+    bank = synth.make_bank(wl, DEV)
+    q_orc = synth.make_q_tables(wl)                      # the oracle's tables
+    mem = make_mem(evk, bank, q_orc, scoring=scoring)
+    bank_bits = host_bits(bank)
+    del bank
+    for rnd in range(4):
         stage = rnd % 2
+        queries = synth.make_queries(wl, b, DEV, salt=rnd)
+        out = run_retrieve(evk, mem, queries, stage, wl.k1, wl.k2, wl.w)
+        # one query in each of the 32 query tiles: the first row of tile 0, the last row of the last
+        # tile, a row of this round's own choice elsewhere
+        sample = tile_sample(b, 1, seed=10 + rnd)
+        sample[-1] = b - 1
+        ep, ef = parity.check_retrieve(bank_bits, host_bits(queries), q_orc[stage], wl.k1, wl.k2, wl.w, out,
+                                       sample=sample, workers=6)
+        parity.record(f"large_compute round {rnd} (stage {stage})", scoring, len(sample), b, ep, ef)
+        assert ep >= 0.9 and ef >= 0.9
         ids, r = synth.make_updates(wl, round_idx=rnd)
         evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), stage, torch.from_numpy(r).to(DEV), wl.alpha)
         got = evk.evk_q_read(mem, stage).cpu().numpy()
-        parity.check_update(q[stage], ids, r, wl.alpha, got)
-        q[stage] = got
-    assert evk.evk_last_status(mem) == 0
+        parity.check_update(q_orc[stage], ids, r, wl.alpha, got)          # whole table, bit for bit
+        q_orc[stage] = oracle.q_update_f32(q_orc[stage], ids, r, wl.alpha)
+        other = evk.evk_q_read(mem, 1 - stage).cpu().numpy()
+        assert np.array_equal(other.view(np.uint32), q_orc[1 - stage].view(np.uint32))
+        assert evk.evk_last_status(mem) == 0
+
+
+def test_retrieved_items_are_updated_and_retrieved_again(evk, scoring):
+    """The method's own loop on one stage: retrieve a context, reward it, update exactly the
+    retrieved items (Eq. 4), retrieve again.  Every later retrieval ranks pools whose values an
+    update wrote.  The oracle follows with its own tables; the ids that get updated on BOTH sides
+    are the oracle's own retrieval (the library's result has just been checked against it), so
+    nothing the library returned flows into an expected value."""
+    n, d, b, k1, k2, w, alpha = 50000, 256, 96, 48, 6, 0.7, 0.25
+    bank = synth.gaussian_unit(n, d, 201, DEV)
+    queries = synth.gaussian_unit(b, d, 202, DEV)          # the same tasks come back every round
+    q_orc = np.random.default_rng(203).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_orc, scoring=scoring)
+    bank_bits, q_bits = host_bits(bank), host_bits(queries)
+    rng = np.random.default_rng(204)
+    moved = 0
+    first_ids = None
+    for rnd in range(6):
+        out = run_retrieve(evk, mem, queries, 1, k1, k2, w)
+        ep, ef = parity.check_retrieve(bank_bits, q_bits, q_orc[1], k1, k2, w, out)
+        assert ep >= 0.9 and ef >= 0.9
+        if first_ids is None:
+            first_ids = out[0].copy()
+        else:
+            moved += int((out[0] != first_ids).any(axis=1).sum())
+        # one reward per query, shared by the k2 items of its context
+        r_q = (rng.random(b) < 0.4).astype(np.float32) * 2 - 1
+        ids = oracle.retrieve(bank_bits, q_bits, q_orc[1], k1, k2, w)[0].reshape(-1).astype(np.int32)
+        r = np.repeat(r_q, k2).astype(np.float32)
+        evk.evk_q_update(mem, torch.from_numpy(ids).to(DEV), 1, torch.from_numpy(r).to(DEV), alpha)
+        got = evk.evk_q_read(mem, 1).cpu().numpy()
+        parity.check_update(q_orc[1], ids, r, alpha, got)
+        q_orc[1] = oracle.q_update_f32(q_orc[1], ids, r, alpha)
+    assert moved > 0          # the updates did change later retrievals
+    parity.record("retrieve-update loop, 6 rounds", scoring, b, b, ep, ef)
 
 
 # ---------------------------------------------------------------------------
@@ -376,6 +450,39 @@ def test_host_buffer_entry_points(evk):
     parity.check_update(q_tab[0], ids.numpy(), r.numpy(), 0.25, evk.evk_q_read(mem, 0).cpu().numpy())
 
 
+def test_host_buffer_calls_check_arguments_before_copying(evk):
+    # a refused call enqueues nothing: no kernel is launched, the outputs keep their contents
+    n, d, b, k1, k2 = 5000, 128, 4, 32, 4
+    bank = synth.gaussian_unit(n, d, 83, DEV)
+    q_tab = np.random.default_rng(6).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab)
+    q_host = synth.gaussian_unit(b, d, 84, "cpu").pin_memory()
+    ids_h = torch.full((b, k2), -7, dtype=torch.int32).pin_memory()
+    sc_h = torch.full((b, k2), -7.0, dtype=torch.float32).pin_memory()
+    before = evk.evk_launch_count(mem)
+    for stage, kk1, kk2, w in ((2, k1, k2, 0.5), (-1, k1, k2, 0.5), (0, k1, k2, 1.5), (0, k1, k2, float("nan")),
+                              (0, k1, k1 + 1, 0.5), (0, 0, 1, 0.5), (0, evk.EVK_MAX_K1 + 1, 1, 0.5)):
+        with pytest.raises(evk.EvkError) as e:
+            evk.evk_retrieve_host(mem, q_host, stage, kk1, kk2, w, ids_h, sc_h)
+        assert e.value.status == evk.EVK_ERR_INVALID
+    ids = torch.arange(10, dtype=torch.int32).pin_memory()
+    r = torch.ones(10).pin_memory()
+    for stage, alpha in ((2, 0.5), (-1, 0.5), (0, 0.0), (0, 1.5), (0, float("nan"))):
+        with pytest.raises(evk.EvkError) as e:
+            evk.evk_q_update_host(mem, ids, stage, r, alpha)
+        assert e.value.status == evk.EVK_ERR_INVALID
+    torch.cuda.synchronize()
+    assert evk.evk_launch_count(mem) == before
+    assert torch.all(ids_h == -7) and torch.all(sc_h == -7.0)
+    assert np.array_equal(evk.evk_q_read(mem, 0).cpu().numpy().view(np.uint32), q_tab[0].view(np.uint32))
+    # a device-detected error still leaves the stream drained and the handle usable
+    bad = torch.tensor([1, n + 5, 2], dtype=torch.int32).pin_memory()
+    evk.evk_q_update_host(mem, bad, 0, torch.ones(3).pin_memory(), 0.5)
+    assert evk.evk_last_status(mem) == evk.EVK_ERR_RANGE
+    evk.evk_retrieve_host(mem, q_host, 0, k1, k2, 0.5, ids_h, sc_h)
+    assert torch.all(ids_h >= 0)
+
+
 def test_both_kernels_return_the_same_pool(evk):
     # the two phase-1 kernels sum in different orders, so similarities may differ in the last
     # bits; the id sets agree except where two entries are within rounding of the boundary
@@ -444,10 +551,12 @@ def test_more_query_tiles_than_sms(evk):
     assert ep >= 0.9 and ef >= 0.9
 
 
-def test_bounded_wait_runs_out_and_the_handle_survives(evk):
+@pytest.mark.parametrize("b", [20, 200, 330])
+def test_bounded_wait_runs_out_and_the_handle_survives(evk, b):
     # failure detection without a fault: the producer of one scan issues no loads, the consumer's
-    # wait expires, every block backs out, and the status word says so
-    n, d, b = 40000, 256, 20
+    # wait expires, every block backs out, and the status word says so.  20 queries: single blocks;
+    # 200: one pair of blocks per tile; 330: a second pair whose other block has a tile of padding
+    n, d = 40000, 256
     bank = synth.gaussian_unit(n, d, 101, DEV)
     queries = synth.gaussian_unit(b, d, 102, DEV)
     q_tab = np.random.default_rng(10).random((2, n)).astype(np.float32)

@@ -130,6 +130,26 @@ def test_phase1_brute_force_against_lexsort():
     assert ids[0, :3].tolist() == [3, 100, 650] and sm[0, 0] == sm[0, 1] == sm[0, 2]
 
 
+def test_rank_step_is_a_lexsort_with_ties_and_padding():
+    # the ranking step taken alone, on similarities with many exact ties
+    rng = np.random.default_rng(70)
+    s = rng.integers(-3, 4, 500).astype(np.float64) / 4.0
+    ids, sm = oracle.rank(s, 120)
+    order = np.lexsort((np.arange(500), -s))[:120]
+    assert ids.tolist() == order.tolist() and np.array_equal(sm, s[order])
+    ids, sm = oracle.rank(s[:7], 10)
+    assert ids[7:].tolist() == [-1] * 3 and np.all(np.isneginf(sm[7:]))
+    assert ids[:7].tolist() == np.lexsort((np.arange(7), -s[:7])).tolist()
+    ids, sm = oracle.rank(np.zeros(0), 3)
+    assert ids.tolist() == [-1] * 3
+    # and phase 1 is exactly sims followed by rank
+    bank = bits_of(rng.standard_normal((300, 24)))
+    q = bits_of(rng.standard_normal(24))
+    a = oracle.phase1(bank, q, 17)
+    b = oracle.rank(oracle.sims(bank, q), 17)
+    assert np.array_equal(a[0][0], b[0]) and np.array_equal(a[1][0], b[1])
+
+
 def test_phase1_k1_equals_size_is_a_permutation_and_padding():
     rng = np.random.default_rng(8)
     bank = bits_of(rng.standard_normal((33, 16)))
