@@ -78,10 +78,13 @@ def retrieve_row_sharded(evk, mem, queries: torch.Tensor, stage: int, k1: int, k
     world = dist.get_world_size(group) if dist.is_initialized() else 1
     if world == 1:
         return evk.evk_merge_shards(gids[None], sims[None], qs[None], k2, w)
-    all_g = torch.empty((world,) + tuple(gids.shape), dtype=gids.dtype, device=gids.device)
-    all_s = torch.empty((world,) + tuple(sims.shape), dtype=sims.dtype, device=sims.device)
-    all_q = torch.empty((world,) + tuple(qs.shape), dtype=qs.dtype, device=qs.device)
-    dist.all_gather_into_tensor(all_g, gids, group=group)
-    dist.all_gather_into_tensor(all_s, sims, group=group)
-    dist.all_gather_into_tensor(all_q, qs, group=group)
-    return evk.evk_merge_shards(all_g, all_s, all_q, k2, w)
+    # gathered along the first axis (rank-major), then viewed as [world][B][k1]
+    b = gids.shape[0]
+    all_g = torch.empty((world * b,) + tuple(gids.shape[1:]), dtype=gids.dtype, device=gids.device)
+    all_s = torch.empty((world * b,) + tuple(sims.shape[1:]), dtype=sims.dtype, device=sims.device)
+    all_q = torch.empty((world * b,) + tuple(qs.shape[1:]), dtype=qs.dtype, device=qs.device)
+    dist.all_gather_into_tensor(all_g, gids.contiguous(), group=group)
+    dist.all_gather_into_tensor(all_s, sims.contiguous(), group=group)
+    dist.all_gather_into_tensor(all_q, qs.contiguous(), group=group)
+    shape = (world,) + tuple(gids.shape)
+    return evk.evk_merge_shards(all_g.view(shape), all_s.view(shape), all_q.view(shape), k2, w)
