@@ -108,6 +108,7 @@ struct MmaParams {
     int sync_tiles;     // kSyncTiles, or kSyncAlways when the scan is bound by HBM and the epilogue has time
     int m64;            // 1 (single block, at most 64 resident queries): M = 64 instructions, half the tensor work
     int stall;          // test aid: the producer of the full scan issues no loads, so a bounded wait runs out
+    int b3d;            // 1: bank stages are kSubRows rows x kSubSlices slices (contiguous bytes per row), see make_map3
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -170,6 +171,21 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
         : "memory");
 }
+// A box of a three-dimensional map {64 columns, rows, 64-column slices}: `rows` x `slices` pieces of
+// 128 bytes, laid down slice by slice as K-major tiles.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int row, int slice) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(row), "r"(slice)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int row, int slice,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(row), "r"(slice), "l"(policy)
+        : "memory");
+}
 // "Evict this first": for data that is read once, so that it does not push out lines that are
 // read again and again (the queries, the histograms, the candidate lists).
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
@@ -193,6 +209,18 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 // M = 64: accumulator row i lands on lane 32 * (i / 16) + i % 16, sixteen rows per lane quarter.
 constexpr uint32_t kInstrDescM64 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
                                    ((uint32_t)(64 >> 4) << 24);
+
+// The contiguous stage layout (resident queries): a stage holds kSubRows bank rows x kSubSlices slices,
+// i.e. 256 contiguous bytes of each row, and feeds N = kSubRows instructions.  Measured over 2 GiB at
+// 1 / 32 / 64 queries: 0.307 / 0.311 / 0.326 ms against 0.314 / 0.317 / 0.330 for 256 rows x 1 slice.
+// 64 rows x 4 slices load faster still (7.3 TB/s) but need four times the instructions, and one
+// tcgen05.mma into an accumulator that the previous one wrote takes ~110 cycles whatever its N: 0.417 ms.
+constexpr int kSubRows = 128;
+constexpr int kSubSlices = 2;
+constexpr uint32_t kInstrDescSub = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSubRows >> 3) << 17) |
+                                   ((uint32_t)(kBlockM >> 4) << 24);
+constexpr uint32_t kInstrDescSubM64 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSubRows >> 3) << 17) |
+                                      ((uint32_t)(64 >> 4) << 24);
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
                                           uint32_t idesc) {
@@ -420,6 +448,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // a width that is no multiple of 64 ends in a partial slice: TMA fills the columns beyond d with
     // zeros, which add nothing to a similarity
     const int k_chunks = (p.d + kBlockK - 1) / kBlockK;
+    // ring stages per bank tile: one per slice, or (contiguous layout) one per (row group, slice group)
+    const int n_sg = (k_chunks + kSubSlices - 1) / kSubSlices;
+    const int n_sub = (!kPair && p.b3d) ? (kBlockN / kSubRows) * n_sg : k_chunks;
     // [resident query tile: k_chunks slices of a_rows x 128 B] [ring of n_stages stages] [barriers]
     const uint32_t a_slice = (uint32_t)p.a_rows * 128u;
     const uint32_t a_region = p.a_resident ? (uint32_t)k_chunks * a_slice : 0u;
@@ -507,10 +538,19 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
                 const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
-                    for (int kc = 0; kc < k_chunks; ++kc) {
+                    for (int u = 0; u < n_sub; ++u) {
                         if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                         const uint32_t s_dst = ring + stage * stage_bytes;
-                        if (kPair) {
+                        if (!kPair && p.b3d) {
+                            // kSubRows rows x kSubSlices slices: each row contributes one contiguous piece
+                            const int row = t * kBlockN + (u / n_sg) * kSubRows, slice = (u % n_sg) * kSubSlices;
+                            mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
+                            if (stream_once)
+                                tma_load_3d_hint(s_dst, &map_bank, full0 + 8 * stage, row, slice, bank_policy);
+                            else
+                                tma_load_3d(s_dst, &map_bank, full0 + 8 * stage, row, slice);
+                        } else if (kPair) {
+                            const int kc = u;
                             // both blocks' bytes are counted on the leader's barrier, which the MMA waits on
                             const uint32_t leader_full = mapa_u32(full0 + 8 * stage, 0);
                             if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * stage, 2 * stage_bytes);
@@ -522,6 +562,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 tma_load_2d_pair(s_dst + b_off, &map_bank, leader_full, kc * kBlockK,
                                                  t * kBlockN + (int)rank * (kBlockN / 2));
                         } else {
+                            const int kc = u;
                             mbar_arrive_expect_tx(full0 + 8 * stage, stage_bytes);
                             if (!p.a_resident) tma_load_2d(s_dst, &map_q, full0 + 8 * stage, kc * kBlockK, qt * kBlockM);
                             if (stream_once)
@@ -547,12 +588,33 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * kBlockN;
-                    for (int kc = 0; kc < k_chunks; ++kc) {
+                    for (int u = 0; u < n_sub; ++u) {
                         if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, wait_limit)) { ok = false; break; }
                         tc_fence_after();
+                        const uint32_t s_addr = ring + stage * stage_bytes;
+                        if (!kPair && p.b3d) {
+                            // this stage: row group g of the tile, slice group sg -> accumulator columns of group g
+                            const int g = u / n_sg, sg = u % n_sg;
+                            const uint32_t idesc = p.m64 ? kInstrDescSubM64 : kInstrDescSub;
+#pragma unroll
+                            for (int sl = 0; sl < kSubSlices; ++sl) {
+                                const int kc = sg * kSubSlices + sl;
+                                if (kc < k_chunks) {
+                                    const uint64_t a_desc = smem_desc(tiles + kc * a_slice);
+                                    const uint64_t b_desc = smem_desc(s_addr + sl * (kSubRows * 128));
+#pragma unroll
+                                    for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                                        umma_bf16(d_tmem + g * kSubRows, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                                  (kc > 0 || k > 0) ? 1u : 0u, idesc);
+                                }
+                            }
+                            umma_commit(empty0 + 8 * stage);
+                            if (++stage == kStages) { stage = 0; phase ^= 1; }
+                            continue;
+                        }
+                        const int kc = u;
                         // a resident query tile narrower than 128 rows is read past its end: the
                         // surplus accumulator rows belong to no query and are never looked at
-                        const uint32_t s_addr = ring + stage * stage_bytes;
                         const uint64_t a_desc = smem_desc(p.a_resident ? tiles + kc * a_slice : s_addr);
                         const uint64_t b_desc = smem_desc(s_addr + b_off);
 #pragma unroll
@@ -1001,6 +1063,23 @@ bool make_map(CUtensorMap *map, const void *base, int d, int64_t rows, int64_t r
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen as {64 columns, rows, slices of 64 columns}, boxed 64 x kSubRows x kSubSlices: one
+// copy brings kSubSlices * 128 contiguous bytes of each row and lays them down as kSubSlices K-major
+// tiles.  (Plain copies into shared memory, measured on B200 over 2 GiB: 7.2 TB/s with 256 contiguous
+// bytes per row, 7.3 with 512, against 6.9-7.0 TB/s for boxes of 256 rows x 128 bytes.)
+// Needs a width that is a multiple of 64: the innermost extent is a fixed 64 columns.
+bool make_map3(CUtensorMap *map, const void *base, int d, int64_t rows, int64_t row_stride_elems) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || d % kBlockK != 0) return false;
+    const cuuint64_t gdim[3] = {(cuuint64_t)kBlockK, (cuuint64_t)rows, (cuuint64_t)(d / kBlockK)};
+    const cuuint64_t gstride[2] = {(cuuint64_t)row_stride_elems * 2, (cuuint64_t)kBlockK * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kSubRows, (cuuint32_t)kSubSlices};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Shared-memory plan for a batch: does the query tile stay resident, how deep is the ring.
 struct SmemPlan {
     int a_resident, a_rows, n_stages;
@@ -1183,11 +1262,15 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.m64 = (sp.a_resident && sp.a_rows <= 64) ? 1 : 0;
     p.a_rows = sp.a_rows;
     p.n_stages = sp.n_stages;
+    // resident queries and a width of whole slices: bank stages of 64 rows x 4 slices
+    p.b3d = (sp.a_resident && d % kBlockK == 0) ? 1 : 0;
 
     if (pl.n_sample) {
         // dense pass over every sample_stride-th row
         CUtensorMap map_sample;
-        if (!make_map(&map_sample, bank, d, pl.n_sample, pl.sample_stride * d, kBlockN)) return cudaErrorInvalidValue;
+        if (!(p.b3d ? make_map3(&map_sample, bank, d, pl.n_sample, pl.sample_stride * d)
+                    : make_map(&map_sample, bank, d, pl.n_sample, pl.sample_stride * d, kBlockN)))
+            return cudaErrorInvalidValue;
         p.size = pl.n_sample;
         p.mode = 1;
         p.n_tiles = pl.n_sample / kBlockN;
@@ -1219,7 +1302,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     }
 
     // in a pair every block loads its half of a bank slice (128 rows) and its own query slice
-    if (!make_map(&map_bank, bank, d, capacity, d, pl.pair ? kBlockN / 2 : kBlockN)) return cudaErrorInvalidValue;
+    if (pl.pair) p.b3d = 0;
+    if (!(p.b3d ? make_map3(&map_bank, bank, d, capacity, d)
+                : make_map(&map_bank, bank, d, capacity, d, pl.pair ? kBlockN / 2 : kBlockN)))
+        return cudaErrorInvalidValue;
     size_t smem_bytes = sp.bytes;
     if (pl.pair) {
         p.m64 = 0;

@@ -386,6 +386,40 @@ def test_update_duplicates_split_and_order(evk):
     parity.check_update(q0, ids, r, 1.0, evk.evk_q_read(mem, 0).cpu().numpy())
 
 
+@pytest.mark.parametrize("m", [2047, 2048, 2049, 9000, 65536, 65537, 150000])
+def test_update_paths_by_batch_length(evk, m):
+    # the single-block kernel (up to 2,048 updates), the one-cluster sort (up to 65,536) and the
+    # multi-launch sort beyond: each at its edges, with a hot id, a run that crosses every block
+    # boundary of the cluster, both step-size rules, and a rejected batch that must change nothing
+    n = 1 << 20
+    rng = np.random.default_rng(m)
+    ids = rng.integers(0, n, m)
+    ids[rng.random(m) < 0.3] = 777777                       # ~30 % of the batch on one entry
+    ids[::97] = 5                                            # and a run spread evenly over the batch
+    ids = ids.astype(np.int32)
+    r = rng.standard_normal(m).astype(np.float32)
+    q0 = rng.standard_normal((2, n)).astype(np.float32)
+    bank = torch.zeros((n, 64), device=DEV, dtype=torch.bfloat16)
+    mem = make_mem(evk, bank, q0)
+    t_ids, t_r = torch.from_numpy(ids).to(DEV), torch.from_numpy(r).to(DEV)
+    bad = t_ids.clone()
+    bad[m - 1] = n
+    evk.evk_q_update(mem, bad, 0, t_r, 0.2)
+    assert evk.evk_last_status(mem) == evk.EVK_ERR_RANGE
+    bad_r = t_r.clone()
+    bad_r[m // 2] = float("inf")
+    evk.evk_q_update(mem, t_ids, 0, bad_r, 0.2)
+    assert evk.evk_last_status(mem) == evk.EVK_ERR_NONFINITE
+    assert np.array_equal(evk.evk_q_read(mem, 0).cpu().numpy().view(np.uint32), q0[0].view(np.uint32))
+    evk.evk_q_update(mem, t_ids, 0, t_r, 0.2)
+    assert evk.evk_last_status(mem) == 0
+    parity.check_update(q0[0], ids, r, 0.2, evk.evk_q_read(mem, 0).cpu().numpy())
+    evk.evk_q_update_decay(mem, t_ids, 1, t_r)
+    want, visits = oracle.q_update_decay(q0[1], np.zeros(n, np.uint32), ids, r)
+    assert np.array_equal(evk.evk_q_read(mem, 1).cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(evk.evk_visits_read(mem, 1).cpu().numpy().view(np.uint32), visits)
+
+
 def test_bad_updates_are_rejected_before_any_write(evk):
     n = 500
     bank = synth.gaussian_unit(n, 64, 61, DEV)

@@ -69,7 +69,7 @@ def test_random_updates(evk, seed):
     rng = np.random.default_rng(2000 + seed)
     for _ in range(12):
         n = int(rng.choice([1, 5, 300, 70000, (1 << 20) + 3]))
-        m = int(rng.choice([0, 1, 63, 1024, 8192, 8193, 20000, 65536, 100000]))
+        m = int(rng.choice([0, 1, 63, 1024, 2048, 2049, 4000, 8192, 8193, 20000, 65536, 65537, 100000]))
         alpha = float(rng.choice([1.0, 0.5, 0.1, 0.05]))
         kind = str(rng.choice(["uniform", "hot", "zipf"]))
         if kind == "uniform":
