@@ -13,6 +13,8 @@ constexpr int kThreads = 256;
 // (the query conversion; inserts use insert_kernel below)
 __global__ void __launch_bounds__(kThreads)
 insert_rows_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int is_bf16, int64_t n_vec) {
+    pdl_trigger();
+    pdl_wait();
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * kThreads) {
         uint4 out;
         if (is_bf16) {
@@ -39,6 +41,8 @@ insert_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int
               float *__restrict__ q_tables, uint32_t *__restrict__ visits, int64_t capacity, int n_stages,
               int64_t first, int64_t n, int stage, const float *__restrict__ q_init, float q_default,
               int32_t *__restrict__ ids_out) {
+    pdl_trigger();
+    pdl_wait();   // the rows may come out of, and the value slots may still be read by, the kernel before
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * kThreads) {
         uint4 out;
         if (is_bf16) {
@@ -83,20 +87,18 @@ cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits
                           cudaStream_t stream, int *launches) {
     if (n <= 0) return cudaSuccess;
     const int64_t n_vec = n * d / 8;
-    insert_kernel<<<grid_for(n_vec > n ? n_vec : n), kThreads, 0, stream>>>(
-        bank + first * d, emb, emb_dtype == EVK_DTYPE_BF16, n_vec, q_tables, visits, capacity, n_stages, first, n,
-        stage, q_init, q_default, ids_out);
     ++*launches;
-    return cudaGetLastError();
+    return launch_overlapped(insert_kernel, dim3(grid_for(n_vec > n ? n_vec : n)), dim3(kThreads), 0, stream,
+                             bank + first * d, emb, (int)(emb_dtype == EVK_DTYPE_BF16), n_vec, q_tables, visits, capacity,
+                             n_stages, first, n, stage, q_init, q_default, ids_out);
 }
 
 cudaError_t launch_convert_queries(const float *src, __nv_bfloat16 *dst, int64_t n_elems,
                                    cudaStream_t stream, int *launches) {
     if (n_elems <= 0) return cudaSuccess;
     const int64_t n_vec = n_elems / 8;
-    insert_rows_kernel<<<grid_for(n_vec), kThreads, 0, stream>>>(dst, src, 0, n_vec);
     ++*launches;
-    return cudaGetLastError();
+    return launch_overlapped(insert_rows_kernel, dim3(grid_for(n_vec)), dim3(kThreads), 0, stream, dst, src, 0, n_vec);
 }
 
 }  // namespace evk

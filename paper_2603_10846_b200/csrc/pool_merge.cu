@@ -48,6 +48,18 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
         tau = 0;
         offs[0] = 0;
     }
+    // The first 32 keys of the first kSpec lists of every warp are fetched before the list lengths are
+    // known (a list's place does not depend on them), so that lengths and keys cost one trip to memory
+    // together.  What lies behind a list's end is read and dropped.
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kSpec = 10;
+    const int warp = tid >> 5, lane = tid & 31;
+    uint64_t spec[kSpec];
+#pragma unroll
+    for (int u = 0; u < kSpec; ++u) {
+        const int p = warp + u * kWarps;
+        spec[u] = (p < nparts && lane < part_stride) ? part_keys[(list0 + (size_t)p * qt_size) * part_stride + lane] : 0;
+    }
     for (int p = tid; p < nparts; p += kThreads) offs[p + 1] = part_counts[list0 + (size_t)p * qt_size];
     __syncthreads();
     if (tid < 32) {
@@ -70,11 +82,21 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
 
     if (total <= kCap) {
         // Everything fits at once: each warp copies whole lists to their places, no search per key.
-        // Four lists per warp and step, their loads issued together; a list longer than a warp
+#pragma unroll
+        for (int u = 0; u < kSpec; ++u) {
+            const int p = warp + u * kWarps;
+            if (p < nparts) {
+                const int first = offs[p], cnt = offs[p + 1] - first;
+                if (lane < cnt) keys[first + lane] = spec[u];
+                if (cnt > 32) {
+                    const uint64_t *src = part_keys + (list0 + (size_t)p * qt_size) * part_stride;
+                    for (int i = 32 + lane; i < cnt; i += 32) keys[first + i] = src[i];
+                }
+            }
+        }
+        // Further lists four per warp and step, their loads issued together; a list longer than a warp
         // finishes in the loop behind.
-        const int warp = tid >> 5, lane = tid & 31;
-        constexpr int kWarps = kThreads / 32;
-        for (int p0 = warp; p0 < nparts; p0 += 4 * kWarps) {
+        for (int p0 = warp + kSpec * kWarps; p0 < nparts; p0 += 4 * kWarps) {
             uint64_t v[4];
             int first[4], cnt[4];
 #pragma unroll

@@ -81,6 +81,17 @@ constexpr size_t kSmemMax = 232448;                  // 227 KB of dynamic shared
 constexpr size_t kSmemFixed = 1024 + 256 + 1536;     // alignment slack + barriers + tracker mailboxes
 constexpr int kHistBins = 64;
 constexpr int kChunk = 32;                           // accumulator columns per tensor-memory load (pick() assumes 32)
+// Self-starting histogram (scans of one query tile).  A similarity's bin is the top 13 bits of its
+// order-preserving bit pattern (sign, exponent, four mantissa bits: sixteen bins to the octave), so
+// every block bins alike without having seen any data; a query's 64 counters cover the window of
+// bins that the first block to finish its first tile anchors one octave above that tile's largest
+// similarity.  Values above the window count in its top bin, values below it in bin 0, which never
+// serves as a threshold: a counter can only under-state how many entries reach its bin's edge.
+constexpr int kAbsShift = 19;
+constexpr int kAbsBins = 1 << (32 - kAbsShift);
+constexpr int kAbsHeadroom = 16;                     // bins between the anchoring maximum and the window's top
+constexpr int kBootBin = kHistBins - 1 - kAbsHeadroom - 16;   // first tile: entries from this window bin up (half the
+                                                     // anchoring maximum) are counted before any is filed
 constexpr int kSyncTiles = 4;                        // tiles of a job whose threshold the epilogue reads itself
 constexpr int kSyncAlways = 1 << 28;                 // ... or every tile: the tracker stays idle
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
@@ -109,6 +120,8 @@ struct MmaParams {
     int m64;            // 1 (single block, at most 64 resident queries): M = 64 instructions, half the tensor work
     int stall;          // test aid: the producer of the full scan issues no loads, so a bounded wait runs out
     int b3d;            // 1: bank stages are kSubRows rows x kSubSlices slices (contiguous bytes per row), see make_map3
+    int abs_hist;       // 1: no sampled thresholds; the shared histogram bins by the similarity's own bits (see kAbsShift)
+    int *anchor;        // [B] abs_hist: lowest bin of each query's histogram window + 1, 0 until the first block sets it
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -475,6 +488,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         reinterpret_cast<volatile unsigned long long *>(reinterpret_cast<unsigned char *>(bars) + 256 + 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool abs_mode = !kPair && p.abs_hist != 0;
     const long long wait_limit = p.stall ? kTimeoutCycles / 16 : kTimeoutCycles;
     pdl_trigger();
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
@@ -661,8 +675,16 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             float h_lo = 0.0f, h_scale = 0.0f;
             int tau_bin = 0;
             unsigned *my_hist = nullptr;
+            // self-starting histogram: window base (in absolute bins), whether this thread has one yet, and
+            // the window bin from which this tile's entries were already counted ahead of filing
+            int a_base = 0, skip_from = kHistBins;
+            bool anchored = false;
             if (q_valid) {
-                if (p.tau0) {
+                if (abs_mode) {
+                    key_sim_floor = -INFINITY;
+                    tau_key = 0;
+                    my_hist = p.hist + (size_t)q * kHistBins;
+                } else if (p.tau0) {
                     // every entry whose similarity reaches the sampled threshold passes
                     key_sim_floor = p.tau0[q];
                     tau_key = (uint64_t)ordered_bits(key_sim_floor + 0.0f) << 32;
@@ -676,7 +698,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 tau_sim = key_sim_floor;
             }
-            slot_q[m] = my_hist ? q : -1;   // the tracker follows this query from now on
+            slot_q[m] = (my_hist && !abs_mode) ? q : -1;   // the tracker follows this query from now on
             int cnt = 0;
             uint64_t *my_buf = p.cand + ((size_t)list_job * kBlockM + (row < 0 ? 0 : row)) * kMmaCandCap;
             // Files one similarity that reached tau_sim.
@@ -685,13 +707,15 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const uint64_t key = make_key(s, (int32_t)row);
                     int bin = 0;
                     if (my_hist) {
-                        // truncation and the clamp at 0 together equal floor and the clamp
-                        bin = __float2int_rz((s - h_lo) * h_scale);
+                        if (abs_mode)
+                            bin = anchored ? (int)(ordered_bits(s + 0.0f) >> kAbsShift) - a_base : 0;
+                        else   // truncation and the clamp at 0 together equal floor and the clamp
+                            bin = __float2int_rz((s - h_lo) * h_scale);
                         bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
                     }
                     if (key > tau_key && bin >= tau_bin) {
                         my_buf[cnt++] = key;
-                        if (my_hist) atomicAdd(my_hist + bin, 1u);
+                        if (my_hist && bin < skip_from && (anchored || !abs_mode)) atomicAdd(my_hist + bin, 1u);
                     }
                 }
             };
@@ -755,9 +779,12 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             auto raise_bin = [&](int best) {
                 if (best > tau_bin) {
                     tau_bin = best;
-                    // a similarity in bin b is at least h_lo + b / h_scale up to rounding; stay a
-                    // hundredth of a bin below that and let the bin test decide
-                    tau_sim = fmaxf(key_sim_floor, h_lo + ((float)tau_bin - 0.01f) / h_scale);
+                    // self-starting: the smallest value of that bin, exactly.  Sampled range: a similarity in
+                    // bin b is at least h_lo + b / h_scale up to rounding; stay a hundredth of a bin below that
+                    // and let the bin test decide
+                    tau_sim = fmaxf(key_sim_floor,
+                                    abs_mode ? from_ordered_bits((uint32_t)(a_base + tau_bin) << kAbsShift)
+                                             : h_lo + ((float)tau_bin - 0.01f) / h_scale);
                 }
             };
             // Takes the tracker's latest word for this query.
@@ -768,47 +795,138 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
             };
             int sync_left = p.sync_tiles;
-            for (int t = split; t < p.n_tiles && ok; t += p.splits) {
-                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
-                tc_fence_after();
-                if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
-                // At the start of a job a threshold moves with every tile and the tracker's word comes
-                // a tile late: there the thread reads its counters itself, later it takes the word.
-                if (sync_left > 0) {
-                    --sync_left;
-                    // (nothing to read before the block's very first tile: every block starts at once
-                    // and the counters are still empty)
-                    if (my_hist && !(job == worker && t == split)) raise_bin(hist_best_bin(my_hist, p.k1));
-                } else {
-                    refresh();
+            // self-starting histogram: the job's first tile is counted when it arrives but filed only when
+            // the second one is there (or the job ends); `held` says that its accumulator is still ours
+            bool held = false;
+            uint32_t held_acc = 0;
+            int64_t held_row0 = 0;
+            for (int t = split; ok; t += p.splits) {
+                const bool real = t < p.n_tiles;
+                if (!real && !held) break;
+                if (real) {
+                    if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
+                    tc_fence_after();
+                    if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
                 }
-                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
-                const int64_t row0 = (int64_t)t * kBlockN;
-                // two register buffers: the next chunk's load is in flight while one is examined
                 uint32_t va[kChunk], vb[kChunk];
-                tmem_ld_issue(t_addr, va);
-                tmem_ld_wait(va);
+                if (real && abs_mode && p.mode == 0 && t == split) {
+                    // The job's first tile starts the histogram off (every lane of the warp walks through this,
+                    // the tensor-memory loads being warp-wide).  The window is anchored by whoever comes first,
+                    // and the tile's entries from window bin kBootBin up are counted.  Filing waits until the
+                    // next tile is in: by then every block has counted its first tile, and the counters give a
+                    // threshold that a few hundred of the 37,888 rows seen so far pass, where one block's own
+                    // 256 rows could justify none.  The tensor cores want this accumulator back only for the
+                    // third tile, whose rows arrive a whole tile later still.
+                    const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
+                    const int64_t row0 = (int64_t)t * kBlockN;
+                    int enc = my_hist ? __ldcg(p.anchor + q) : 1;
+                    if (__any_sync(0xffffffffu, enc == 0)) {
+                        // nobody has anchored this query's window yet: this tile's largest similarity does
+                        float mx = -INFINITY;
 #pragma unroll 1
-                for (int c0 = 0; c0 < kBlockN - 2 * kChunk; c0 += 2 * kChunk) {
-                    tmem_ld_issue(t_addr + c0 + kChunk, vb);
-                    process(va, row0, c0);
-                    tmem_ld_wait(vb);
-                    tmem_ld_issue(t_addr + c0 + 2 * kChunk, va);
-                    refresh();
-                    process(vb, row0, c0 + kChunk);
+                        for (int c0 = 0; c0 < kBlockN; c0 += kChunk) {
+                            tmem_ld_issue(t_addr + c0, va);
+                            tmem_ld_wait(va);
+#pragma unroll
+                            for (int j = 0; j < kChunk; ++j) {
+                                const float x = __uint_as_float(va[j]);
+                                if (row0 + c0 + j < p.size && fabsf(x) <= 3.0e38f) mx = fmaxf(mx, x);
+                            }
+                        }
+                        if (my_hist && enc == 0 && mx > -INFINITY) {
+                            int prop = (int)(ordered_bits(mx + 0.0f) >> kAbsShift) + kAbsHeadroom - (kHistBins - 1);
+                            prop = prop < 0 ? 0 : (prop > kAbsBins - kHistBins ? kAbsBins - kHistBins : prop);
+                            const int got = atomicCAS(p.anchor + q, 0, prop + 1);
+                            enc = got ? got : prop + 1;
+                        }
+                    }
+                    if (my_hist && enc != 0) {
+                        a_base = enc - 1;
+                        anchored = true;
+                    }
+                    tmem_ld_issue(t_addr, va);
                     tmem_ld_wait(va);
+                    const float cnt_edge = anchored ? from_ordered_bits((uint32_t)(a_base + kBootBin) << kAbsShift) : INFINITY;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kBlockN; c0 += kChunk) {
+                        if (c0 > 0) {
+                            tmem_ld_issue(t_addr + c0, va);
+                            tmem_ld_wait(va);
+                        }
+                        uint32_t bits[kChunk];
+#pragma unroll
+                        for (int j = 0; j < kChunk; ++j) bits[j] = __uint_as_float(va[j]) >= cnt_edge ? (1u << j) : 0u;
+#pragma unroll
+                        for (int w = kChunk / 2; w >= 1; w >>= 1) {
+#pragma unroll
+                            for (int j = 0; j < w; ++j) bits[j] |= bits[j + w];
+                        }
+                        uint32_t pass = bits[0];
+                        while (pass) {
+                            const int j = __ffs(pass) - 1;
+                            pass &= pass - 1;
+                            if (anchored && row0 + c0 + j < p.size) {
+                                int bin = (int)(ordered_bits(__uint_as_float(pick(va, j)) + 0.0f) >> kAbsShift) - a_base;
+                                bin = bin > kHistBins - 1 ? kHistBins - 1 : bin;
+                                atomicAdd(my_hist + bin, 1u);
+                            }
+                        }
+                    }
+                    held = true;
+                    held_acc = acc;
+                    held_row0 = row0;
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                    continue;
                 }
-                tmem_ld_issue(t_addr + kBlockN - kChunk, vb);
-                process(va, row0, kBlockN - 2 * kChunk);
-                tmem_ld_wait(vb);
-                // every column of this accumulator is in registers: hand it back before the last look
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * acc, 0)); else mbar_arrive(tempty0 + 8 * acc);
+                // the tile held back first (if any), then the one that has just arrived (if any)
+#pragma unroll 1
+                for (int rep = held ? 0 : 1; rep < (real ? 2 : 1); ++rep) {
+                    const bool old = rep == 0;
+                    const uint32_t use_acc = old ? held_acc : acc;
+                    const int64_t row0 = old ? held_row0 : (int64_t)t * kBlockN;
+                    // entries of the held tile from kBootBin up are in the counters already
+                    skip_from = (old && anchored) ? kBootBin : kHistBins;
+                    // At the start of a job a threshold moves with every tile and the tracker's word comes
+                    // a tile late: there the thread reads its counters itself, later it takes the word.
+                    if (sync_left > 0) {
+                        if (!old) --sync_left;
+                        // (sampled thresholds: nothing to read before the block's very first tile, every block
+                        // starts at once and the counters are still empty)
+                        if (my_hist && (abs_mode ? anchored : !(job == worker && t == split)))
+                            raise_bin(hist_best_bin(my_hist, p.k1));
+                    } else {
+                        refresh();
+                    }
+                    const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + use_acc * kBlockN;
+                    // two register buffers: the next chunk's load is in flight while one is examined
+                    tmem_ld_issue(t_addr, va);
+                    tmem_ld_wait(va);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kBlockN - 2 * kChunk; c0 += 2 * kChunk) {
+                        tmem_ld_issue(t_addr + c0 + kChunk, vb);
+                        process(va, row0, c0);
+                        tmem_ld_wait(vb);
+                        tmem_ld_issue(t_addr + c0 + 2 * kChunk, va);
+                        refresh();
+                        process(vb, row0, c0 + kChunk);
+                        tmem_ld_wait(va);
+                    }
+                    tmem_ld_issue(t_addr + kBlockN - kChunk, vb);
+                    process(va, row0, kBlockN - 2 * kChunk);
+                    tmem_ld_wait(vb);
+                    // every column of this accumulator is in registers: hand it back before the last look
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * use_acc, 0)); else mbar_arrive(tempty0 + 8 * use_acc);
+                    }
+                    if (!old) {
+                        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                    }
+                    process(vb, row0, kBlockN - kChunk);
                 }
-                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-                process(vb, row0, kBlockN - kChunk);
+                held = false;
+                if (!real) break;
             }
             if (p.mode == 0 && ok && qt < p.n_qt && row >= 0) p.cand_cnt[(size_t)list_job * kBlockM + row] = cnt;
         }
@@ -913,6 +1031,16 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tc_fence_after();
         if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
     }
+}
+
+// Clears the shared histograms and window anchors of a scan that starts them off itself.
+__global__ void __launch_bounds__(256)
+hist_reset_kernel(unsigned *__restrict__ hist, int *__restrict__ anchor, int n_queries) {
+    pdl_trigger();
+    pdl_wait();   // the previous user of this workspace may still be reading them
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i < n_queries * kHistBins) hist[i] = 0;
+    if (i < n_queries) anchor[i] = 0;
 }
 
 // A starting threshold per query from its sample similarities: any value that at least k1 of
@@ -1210,7 +1338,8 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     }
     if (pl.grid < 1) pl.grid = 1;
     // a strided sample of the bank gives each query a starting threshold
-    pl.n_sample = (size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
+    // (scans of one query tile start their thresholds off themselves, see kAbsShift)
+    pl.n_sample = (pl.pair && size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
     pl.sample_stride = pl.n_sample ? size / pl.n_sample : 0;
     pl.stall = 0;
     return pl;
@@ -1251,6 +1380,8 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.tau0 = nullptr;
     p.range = range;
     p.hist = hist;
+    p.abs_hist = pl.pair ? 0 : 1;
+    p.anchor = reinterpret_cast<int *>(tau0);   // the sampled thresholds' array, unused by such a scan
     // One query tile: the scan runs at HBM speed, a bank tile arrives every ~11 us and the epilogue
     // idles most of that, so it reads its counters itself before every tile (freshest thresholds).
     // More tiles: the tensor cores set the pace and the reads move to the tracker warp.
@@ -1321,10 +1452,17 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.n_tiles = pl.n_tiles;
     p.splits = pl.splits;
     cudaError_t err = cudaSuccess;
+    if (p.abs_hist) {
+        const int n = B * kHistBins;
+        err = launch_overlapped(hist_reset_kernel, dim3((n + 255) / 256), dim3(256), 0, stream, hist, p.anchor, B);
+        if (err != cudaSuccess) return err;
+        ++*launches;
+    }
     if (ev_start) err = cudaEventRecord(ev_start, stream);
-    // behind the threshold kernel the scan may start early; its epilogue waits for the thresholds
+    // behind the threshold (or reset) kernel the scan may start early; its epilogue waits for that kernel
     if (err == cudaSuccess)
-        err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, pl.n_sample != 0 && !ev_start, pl.pair != 0, stream);
+        err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, (pl.n_sample != 0 || p.abs_hist) && !ev_start,
+                            pl.pair != 0, stream);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);
