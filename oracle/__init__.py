@@ -54,6 +54,8 @@ def _load():
     lib.evk_oracle_sims.restype = None
     lib.evk_oracle_rank.argtypes = [p, c_i64, c_i32, p, p]
     lib.evk_oracle_rank.restype = c_i32
+    lib.evk_oracle_rank_live.argtypes = [p, p, c_i64, c_i32, p, p]
+    lib.evk_oracle_rank_live.restype = c_i32
     lib.evk_oracle_phase1.argtypes = [p, c_i64, c_i32, p, c_i32, p, p]
     lib.evk_oracle_phase1.restype = c_i32
     lib.evk_oracle_phase2.argtypes = [p, p, c_i32, p, c_f64, c_i32, p, p]
@@ -125,19 +127,25 @@ def sims(bank_bits, query_bits) -> np.ndarray:
     return out
 
 
-def rank(sims_row, k1: int):
+def rank(sims_row, k1: int, live=None):
     """The ranking step of phase 1 on one query's similarities (entry id = index): the first k1
-    by (similarity desc, id asc) after a full sort.  ids int32 [k1], sims fp64 [k1]."""
+    by (similarity desc, id asc) after a full sort.  live (uint8 per entry, optional): entries
+    marked 0 have been dropped from the memory and are left out.  ids int32 [k1], sims fp64 [k1]."""
     sims_row = _c(sims_row, np.float64)
     assert sims_row.ndim == 1
     ids = np.empty(k1, dtype=np.int32)
     sm = np.empty(k1, dtype=np.float64)
-    _load().evk_oracle_rank(_ptr(sims_row), sims_row.size, k1, _ptr(ids), _ptr(sm))
+    if live is None:
+        _load().evk_oracle_rank(_ptr(sims_row), sims_row.size, k1, _ptr(ids), _ptr(sm))
+    else:
+        live = _c(live, np.uint8)
+        assert live.shape == sims_row.shape
+        _load().evk_oracle_rank_live(_ptr(sims_row), _ptr(live), sims_row.size, k1, _ptr(ids), _ptr(sm))
     return ids, sm
 
 
-def phase1(bank_bits, query_bits, k1: int):
-    """Top-k1 pool per query by (similarity desc, id asc): ids int32, sims fp64."""
+def phase1(bank_bits, query_bits, k1: int, live=None):
+    """Top-k1 pool per query by (similarity desc, id asc): ids int32, sims fp64.  live: see rank."""
     bank_bits = _c(bank_bits, np.uint16)
     query_bits = _c(query_bits, np.uint16)
     if query_bits.ndim == 1:
@@ -149,8 +157,11 @@ def phase1(bank_bits, query_bits, k1: int):
     sm = np.empty((b, k1), dtype=np.float64)
     lib = _load()
     for i in range(b):
-        lib.evk_oracle_phase1(_ptr(bank_bits), size, d, _ptr(query_bits[i]), k1,
-                              _ptr(ids[i]), _ptr(sm[i]))
+        if live is None:
+            lib.evk_oracle_phase1(_ptr(bank_bits), size, d, _ptr(query_bits[i]), k1,
+                                  _ptr(ids[i]), _ptr(sm[i]))
+        else:
+            ids[i], sm[i] = rank(sims(bank_bits, query_bits[i]) if size else np.zeros(0), k1, live)
     return ids, sm
 
 
@@ -172,9 +183,9 @@ def phase2(pool_ids, pool_sims, q_stage, w: float, k2: int, zscore: bool = False
     return ids, sc
 
 
-def retrieve(bank_bits, query_bits, q_stage, k1: int, k2: int, w: float, zscore: bool = False):
-    """Both phases; returns (ids, scores, pool_ids, pool_sims)."""
-    pool_ids, pool_sims = phase1(bank_bits, query_bits, k1)
+def retrieve(bank_bits, query_bits, q_stage, k1: int, k2: int, w: float, zscore: bool = False, live=None):
+    """Both phases; returns (ids, scores, pool_ids, pool_sims).  live: see rank."""
+    pool_ids, pool_sims = phase1(bank_bits, query_bits, k1, live)
     ids, sc = phase2(pool_ids, pool_sims, q_stage, w, k2, zscore)
     return ids, sc, pool_ids, pool_sims
 

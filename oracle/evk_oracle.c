@@ -99,19 +99,32 @@ static int ranked_cmp(const void *a, const void *b) {
 }
 
 /* Ranking step of the candidate pool: the `size` similarities sims[] (entry id = index) are
- * fully sorted by (similarity descending, id ascending); the first min(k1, size) are the
- * pool.  Unused slots get id -1 and similarity -inf.  Returns the pool length. */
-int32_t evk_oracle_rank(const double *sims, int64_t size, int32_t k1,
-                        int32_t *pool_ids, double *pool_sims) {
-    int32_t n_pool = (int32_t)((int64_t)k1 < size ? (int64_t)k1 : size);
+ * fully sorted by (similarity descending, id ascending); the first min(k1, n_live) are the
+ * pool.  live[] (may be NULL: every entry is live) marks entries that have been dropped from
+ * the memory with 0: a dropped entry is simply not there (it takes no place in the order and
+ * cannot be returned), while the ids of the others stay what they were.  Unused slots get id -1
+ * and similarity -inf.  Returns the pool length. */
+int32_t evk_oracle_rank_live(const double *sims, const uint8_t *live, int64_t size, int32_t k1,
+                             int32_t *pool_ids, double *pool_sims) {
     for (int32_t j = 0; j < k1; ++j) { pool_ids[j] = -1; pool_sims[j] = -INFINITY; }
     if (size <= 0) return 0;
     ranked_t *r = (ranked_t *)malloc((size_t)size * sizeof(ranked_t));
-    for (int64_t i = 0; i < size; ++i) { r[i].key = sims[i]; r[i].key2 = 0.0; r[i].id = (int32_t)i; }
-    qsort(r, (size_t)size, sizeof(ranked_t), ranked_cmp);
+    int64_t n = 0;
+    for (int64_t i = 0; i < size; ++i) {
+        if (live && !live[i]) continue;
+        r[n].key = sims[i]; r[n].key2 = 0.0; r[n].id = (int32_t)i;
+        ++n;
+    }
+    qsort(r, (size_t)n, sizeof(ranked_t), ranked_cmp);
+    int32_t n_pool = (int32_t)((int64_t)k1 < n ? (int64_t)k1 : n);
     for (int32_t j = 0; j < n_pool; ++j) { pool_ids[j] = r[j].id; pool_sims[j] = r[j].key; }
     free(r);
     return n_pool;
+}
+
+int32_t evk_oracle_rank(const double *sims, int64_t size, int32_t k1,
+                        int32_t *pool_ids, double *pool_sims) {
+    return evk_oracle_rank_live(sims, NULL, size, k1, pool_ids, pool_sims);
 }
 
 /* The top-K candidate pool C(x): every stored entry's similarity (evk_oracle_sims), then the

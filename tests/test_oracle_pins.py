@@ -150,6 +150,43 @@ def test_rank_step_is_a_lexsort_with_ties_and_padding():
     assert np.array_equal(a[0][0], b[0]) and np.array_equal(a[1][0], b[1])
 
 
+def test_dropped_entries_equal_retrieval_on_the_compacted_bank():
+    # Dropping entries from the memory is the same as never having stored them: retrieval over
+    # the bank with a live mask equals retrieval over the bank with those rows removed, once the
+    # compacted ids are mapped back.  (Exact ties included: rows 3, 100 and 650 are one vector.)
+    rng = np.random.default_rng(71)
+    n, d, k1, k2 = 700, 40, 50, 6
+    bank = bits_of(rng.standard_normal((n, d)))
+    bank[100] = bank[3]
+    bank[650] = bank[3]
+    qs = np.concatenate([bits_of(rng.standard_normal((4, d))), bank[3:4]])
+    q_stage = rng.random(n).astype(np.float32)
+    live = (rng.random(n) < 0.6).astype(np.uint8)
+    live[3], live[100], live[650] = 1, 0, 1          # the middle copy of the tie is gone
+    kept = np.nonzero(live)[0]
+    got = oracle.retrieve(bank, qs, q_stage, k1, k2, 0.4, live=live)
+    want = oracle.retrieve(bank[kept], qs, q_stage[kept], k1, k2, 0.4)
+    assert np.array_equal(got[2], kept[want[2]]) and np.array_equal(got[3], want[3])
+    assert np.array_equal(got[0], kept[want[0]]) and np.array_equal(got[1], want[1])
+    assert got[2][4, :2].tolist() == [3, 650]          # the query equal to the tied rows: 100 is skipped
+    # nothing dropped: the plain retrieval; everything dropped: padding only; fewer live than k1
+    all_live = oracle.retrieve(bank, qs, q_stage, k1, k2, 0.4, live=np.ones(n, np.uint8))
+    plain = oracle.retrieve(bank, qs, q_stage, k1, k2, 0.4)
+    assert all(np.array_equal(a, b) for a, b in zip(all_live, plain))
+    none = oracle.phase1(bank, qs[0], 5, live=np.zeros(n, np.uint8))
+    assert none[0].tolist() == [[-1] * 5] and np.all(np.isneginf(none[1]))
+    few = np.zeros(n, np.uint8)
+    few[[9, 500, 77]] = 1
+    ids, sm = oracle.phase1(bank, qs[1], 8, live=few)
+    assert sorted(ids[0, :3].tolist()) == [9, 77, 500] and ids[0, 3:].tolist() == [-1] * 5
+    # the ranking step alone, against a lexsort restricted to the live entries
+    s = rng.integers(-3, 4, 300).astype(np.float64)
+    lv = (rng.random(300) < 0.5).astype(np.uint8)
+    ids, sm = oracle.rank(s, 40, live=lv)
+    order = [i for i in np.lexsort((np.arange(300), -s)) if lv[i]][:40]
+    assert ids.tolist() == order and np.array_equal(sm, s[order])
+
+
 def test_phase1_k1_equals_size_is_a_permutation_and_padding():
     rng = np.random.default_rng(8)
     bank = bits_of(rng.standard_normal((33, 16)))
