@@ -72,8 +72,9 @@ typedef struct evk_config {
 } evk_config;
 
 /* Bytes of device memory a bank of this shape needs (embeddings as bf16 rows
- * [capacity][d], value tables fp32 and update counts uint32 [n_stages][capacity], a status word).  0 if the
- * config is invalid.  `arena` and `arena_bytes` are ignored. */
+ * [capacity][d], value tables fp32 and update counts uint32 [n_stages][capacity], one live bit per
+ * entry, a block of status and counter words).  0 if the config is invalid.  `arena` and `arena_bytes`
+ * are ignored. */
 size_t evk_mem_bytes_required(const evk_config *cfg);
 
 /* Create an empty memory M_0 over the caller's arena (Eq. 1 starts from a seed
@@ -212,6 +213,45 @@ int evk_q_write(evk_mem *mem, int stage, int64_t first, int64_t n, const float *
 
 /* Copy the stored bf16 rows [first .. first+n) to a device array [n][d] of uint16. */
 int evk_bank_read(evk_mem *mem, int64_t first, int64_t n, void *out_bf16, void *stream);
+
+/* Dropping entries from a live memory.  The memory of Eq. 1 only grows, but the method also hands
+ * a FILTERED bank on (Experiment section, transfer across backbones: a bank from which entries were
+ * removed initialises another generator's run), so entries can be taken out without rebuilding the
+ * bank.  Every id in ids [n] (device) loses its place: no retrieval on this stream after this call
+ * returns it, it takes no slot of a pool, and evk_select_by_value skips it.  The other entries keep
+ * their ids; the dropped entry's row and values stay in the arena (an update that names it is
+ * applied and never seen).  Naming an id twice, or one that was dropped before, is harmless.  If
+ * any id is outside [0, size) the whole call does nothing and the status word becomes EVK_ERR_RANGE.
+ * A pool is then as long as min(k1, live entries).  There is no way to bring an entry back. */
+int evk_mem_tombstone(evk_mem *mem, const int32_t *ids, int64_t n, void *stream);
+
+/* Carrying a memory from one run into the next (Experiment section: the bank learned on one level
+ * of tasks initialises the run on the next; a bank is handed to other generators).
+ * evk_mem_export copies entries [first, first + n) out to caller buffers on the device, any of
+ * which may be NULL: rows_bf16 [n][d] (uint16 bit patterns), q [n_stages][n], visits
+ * [n_stages][n] (the counts of evk_q_update_decay), live [n] (1 = in the memory, 0 = dropped).
+ * evk_mem_import appends n entries from such buffers: rows are required; NULL q / visits / live
+ * mean q_default / 0 / all live.  Entries marked 0 in `live` keep their place (ids are positions)
+ * but are dropped at once; a caller that wants a compact bank leaves them out of the buffers.
+ * ids_out [n] (may be NULL) receives the new ids.  Errors: EVK_ERR_INVALID (range, null rows),
+ * EVK_ERR_CAPACITY (nothing is imported). */
+int evk_mem_export(evk_mem *mem, int64_t first, int64_t n, void *rows_bf16, float *q, uint32_t *visits,
+                   uint8_t *live, void *stream);
+int evk_mem_import(evk_mem *mem, int64_t n, const void *rows_bf16, const float *q, const uint32_t *visits,
+                   const uint8_t *live, int32_t *ids_out, void *stream);
+
+/* Counters of one bank (no counterpart in the paper: they explain a slow batch in the field).
+ * Synchronises `stream`.  candidates_filed: (similarity, id) pairs the tensor-core scans left in
+ * their candidate lists for the merge, summed over all retrievals (k1 per query is the least
+ * possible); list_cutbacks: times such a list filled up and was cut back to its best k1 (only
+ * adversarial row orders cause it); longest_update_run: the most updates one entry received in a
+ * single batch (runs of more than 8), which one thread or warp has to apply one after another. */
+typedef struct evk_stats {
+    int64_t entries, live_entries, dropped_entries;
+    int64_t retrieve_calls, update_calls, insert_calls, kernel_launches;
+    int64_t candidates_filed, list_cutbacks, longest_update_run;
+} evk_stats;
+int evk_mem_stats(evk_mem *mem, evk_stats *out, void *stream);
 
 /* Host-buffer forms of the two hot calls, for callers whose data lives in host
  * memory (pinned memory makes the copies asynchronous).  They copy the inputs to

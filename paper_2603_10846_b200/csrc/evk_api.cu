@@ -35,7 +35,11 @@ struct evk_mem {
     __nv_bfloat16 *bank;  // [capacity][d]
     float *q_tables;      // [n_stages][capacity]
     uint32_t *visits;     // [n_stages][capacity] updates received (decreasing step size)
-    int32_t *status;      // device status word
+    uint32_t *live_bits;  // [ceil(capacity / 32)] one bit per entry: 1 = in the memory, 0 = dropped
+    int32_t *status;      // device status word (word 0 of the device block)
+    uint32_t *dev;        // the device block as words: live count, counters (see DevWord)
+    int any_dropped;      // an entry may have been dropped: the scans consult the live bits
+    int64_t n_retrieve, n_update, n_insert;   // calls that enqueued work
     int scoring;
     int score_norm;       // EVK_NORM_*: how phase 2 mixes similarity and value
     int stall_next;       // evk_mem_inject_stall: the next tensor-path retrieve starves its consumer
@@ -48,7 +52,7 @@ namespace {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct ArenaLayout {
-    size_t bank, q_tables, visits, status, total;
+    size_t bank, q_tables, visits, live_bits, status, total;
 };
 
 bool config_ok(const evk_config *c) {
@@ -62,7 +66,8 @@ ArenaLayout arena_layout(const evk_config *c) {
     l.bank = 0;
     l.q_tables = align256((size_t)c->capacity * c->d * sizeof(__nv_bfloat16));
     l.visits = l.q_tables + align256((size_t)c->n_stages * c->capacity * sizeof(float));
-    l.status = l.visits + align256((size_t)c->n_stages * c->capacity * sizeof(uint32_t));
+    l.live_bits = l.visits + align256((size_t)c->n_stages * c->capacity * sizeof(uint32_t));
+    l.status = l.live_bits + align256((size_t)((c->capacity + 31) / 32) * sizeof(uint32_t));
     l.total = l.status + 256;
     return l;
 }
@@ -136,7 +141,11 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     m->bank = reinterpret_cast<__nv_bfloat16 *>(base + l.bank);
     m->q_tables = reinterpret_cast<float *>(base + l.q_tables);
     m->visits = reinterpret_cast<uint32_t *>(base + l.visits);
+    m->live_bits = reinterpret_cast<uint32_t *>(base + l.live_bits);
     m->status = reinterpret_cast<int32_t *>(base + l.status);
+    m->dev = reinterpret_cast<uint32_t *>(base + l.status);
+    m->any_dropped = 0;
+    m->n_retrieve = m->n_update = m->n_insert = 0;
     m->scoring = EVK_SCORING_AUTO;
     m->score_norm = EVK_NORM_NONE;
     m->stall_next = 0;
@@ -187,12 +196,13 @@ int evk_mem_insert(evk_mem *mem, const void *emb, int emb_dtype, int64_t n, int 
     if (!emb || !aligned(emb, 16)) return EVK_ERR_INVALID;
     if (mem->size + n > mem->cfg.capacity) return EVK_ERR_CAPACITY;
     int launches = 0;
-    cudaError_t err = launch_insert(mem->bank, mem->q_tables, mem->visits, mem->cfg.capacity, mem->cfg.d,
+    cudaError_t err = launch_insert(mem->bank, mem->q_tables, mem->visits, mem->live_bits, mem->dev, mem->cfg.capacity, mem->cfg.d,
                                     mem->cfg.n_stages, mem->size, n, emb, emb_dtype, stage, q_init,
                                     mem->cfg.q_default, ids_out, static_cast<cudaStream_t>(stream), &launches);
     mem->launches += launches;
     if (err != cudaSuccess) return EVK_ERR_CUDA;
     mem->size += n;
+    ++mem->n_insert;
     return EVK_OK;
 }
 
@@ -242,6 +252,8 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
             MmaPlan plan = mma_plan(mem->size, B, k1);
             plan.stall = mem->stall_next;
             mem->stall_next = 0;
+            plan.live_bits = mem->any_dropped ? mem->live_bits : nullptr;
+            plan.dev = mem->dev;
             uint64_t *cand = nullptr;
             int *cand_cnt = nullptr;
             err = launch_score_mma(mem->bank, mem->size, mem->cfg.capacity, mem->cfg.d, q_bf16, B, k1, plan,
@@ -252,7 +264,8 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
             part_stride = kMmaCandCap;
             qt_size = 128;
         } else {
-            const StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+            StreamPlan plan = stream_plan(mem->size, mem->cfg.d, B, k1);
+            plan.live_bits = mem->any_dropped ? mem->live_bits : nullptr;
             uint64_t *keys = reinterpret_cast<uint64_t *>(ws + l.part_keys);
             int *counts = reinterpret_cast<int *>(ws + l.part_counts);
             if (ev_start) err = cudaEventRecord(ev_start, stream);
@@ -267,11 +280,13 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
     }
     const int expect = (int)(mem->size < k1 ? mem->size : k1);
     if (err == cudaSuccess)
-        err = launch_merge_rerank(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect, mem->status,
+        err = launch_merge_rerank(part_keys, part_counts, nparts, part_stride, qt_size, B, k1, expect,
+                                  mem->any_dropped ? mem->dev + kDevLive : nullptr, mem->status,
                                   pool_ids_out, pool_sims_out, k2,
                                   mem->q_tables + (size_t)stage * mem->cfg.capacity, w, mem->score_norm, ids_out,
                                   scores_out, stream, &launches);
     mem->launches += launches;
+    ++mem->n_retrieve;
     return cuda_status(err);
 }
 
@@ -315,8 +330,9 @@ int evk_q_update(evk_mem *mem, const int32_t *ids, int64_t M, int stage,
     int launches = 0;
     cudaError_t err = launch_q_update(mem->q_tables + (size_t)stage * mem->cfg.capacity, mem->size, ids, rewards,
                                       M, alpha, nullptr, mem->status, workspace, static_cast<cudaStream_t>(stream),
-                                      &launches);
+                                      &launches, mem->dev + kDevLongestRun);
     mem->launches += launches;
+    ++mem->n_update;
     return cuda_status(err);
 }
 
@@ -330,8 +346,10 @@ int evk_q_update_decay(evk_mem *mem, const int32_t *ids, int64_t M, int stage, c
     int launches = 0;
     const size_t off = (size_t)stage * mem->cfg.capacity;
     cudaError_t err = launch_q_update(mem->q_tables + off, mem->size, ids, rewards, M, 1.0f, mem->visits + off,
-                                      mem->status, workspace, static_cast<cudaStream_t>(stream), &launches);
+                                      mem->status, workspace, static_cast<cudaStream_t>(stream), &launches,
+                                      mem->dev + kDevLongestRun);
     mem->launches += launches;
+    ++mem->n_update;
     return cuda_status(err);
 }
 
@@ -393,6 +411,94 @@ int evk_bank_read(evk_mem *mem, int64_t first, int64_t n, void *out_bf16, void *
     return cuda_status(cudaMemcpyAsync(out_bf16, mem->bank + (size_t)first * mem->cfg.d,
                                        (size_t)n * mem->cfg.d * sizeof(__nv_bfloat16), cudaMemcpyDeviceToDevice,
                                        static_cast<cudaStream_t>(stream)));
+}
+
+// ---- dropping entries, export, import, counters ------------------------------------------------
+
+int evk_mem_tombstone(evk_mem *mem, const int32_t *ids, int64_t n, void *stream) {
+    if (!mem || n < 0) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!ids) return EVK_ERR_INVALID;
+    int launches = 0;
+    cudaError_t err = launch_tombstone(ids, n, mem->size, mem->live_bits, mem->dev, mem->status,
+                                       static_cast<cudaStream_t>(stream), &launches);
+    mem->launches += launches;
+    mem->any_dropped = 1;
+    return cuda_status(err);
+}
+
+int evk_mem_export(evk_mem *mem, int64_t first, int64_t n, void *rows_bf16, float *q, uint32_t *visits,
+                   uint8_t *live, void *stream_v) {
+    if (!mem || first < 0 || n < 0 || first + n > mem->size) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t err = cudaSuccess;
+    if (rows_bf16)
+        err = cudaMemcpyAsync(rows_bf16, mem->bank + (size_t)first * mem->cfg.d,
+                              (size_t)n * mem->cfg.d * sizeof(__nv_bfloat16), cudaMemcpyDeviceToDevice, stream);
+    for (int s = 0; s < mem->cfg.n_stages && err == cudaSuccess; ++s) {
+        const size_t off = (size_t)s * mem->cfg.capacity + first;
+        if (q)
+            err = cudaMemcpyAsync(q + (size_t)s * n, mem->q_tables + off, (size_t)n * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, stream);
+        if (visits && err == cudaSuccess)
+            err = cudaMemcpyAsync(visits + (size_t)s * n, mem->visits + off, (size_t)n * sizeof(uint32_t),
+                                  cudaMemcpyDeviceToDevice, stream);
+    }
+    int launches = 0;
+    if (live && err == cudaSuccess) err = launch_live_export(mem->live_bits, first, n, live, stream, &launches);
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+int evk_mem_import(evk_mem *mem, int64_t n, const void *rows_bf16, const float *q, const uint32_t *visits,
+                   const uint8_t *live, int32_t *ids_out, void *stream_v) {
+    if (!mem || n < 0) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!rows_bf16 || !aligned(rows_bf16, 16)) return EVK_ERR_INVALID;
+    if (mem->size + n > mem->cfg.capacity) return EVK_ERR_CAPACITY;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int64_t first = mem->size;
+    // the rows go in like any insert (every stage at q_default, counts at 0, live) ...
+    int rc = evk_mem_insert(mem, rows_bf16, EVK_DTYPE_BF16, n, EVK_STAGE_ALL, nullptr, ids_out, stream_v);
+    if (rc != EVK_OK) return rc;
+    // ... then the saved values, update counts and dropped marks are laid over them
+    cudaError_t err = cudaSuccess;
+    for (int s = 0; s < mem->cfg.n_stages && err == cudaSuccess; ++s) {
+        const size_t off = (size_t)s * mem->cfg.capacity + first;
+        if (q)
+            err = cudaMemcpyAsync(mem->q_tables + off, q + (size_t)s * n, (size_t)n * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, stream);
+        if (visits && err == cudaSuccess)
+            err = cudaMemcpyAsync(mem->visits + off, visits + (size_t)s * n, (size_t)n * sizeof(uint32_t),
+                                  cudaMemcpyDeviceToDevice, stream);
+    }
+    int launches = 0;
+    if (live && err == cudaSuccess) {
+        err = launch_live_import(live, first, n, mem->live_bits, mem->dev, stream, &launches);
+        mem->any_dropped = 1;
+    }
+    mem->launches += launches;
+    return cuda_status(err);
+}
+
+int evk_mem_stats(evk_mem *mem, evk_stats *out, void *stream_v) {
+    if (!mem || !out) return EVK_ERR_INVALID;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (cudaMemcpyAsync(w, mem->dev, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return EVK_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return EVK_ERR_CUDA;
+    out->entries = mem->size;
+    out->live_entries = (int64_t)w[kDevLive];
+    out->dropped_entries = (int64_t)w[kDevDropped];
+    out->retrieve_calls = mem->n_retrieve;
+    out->update_calls = mem->n_update;
+    out->insert_calls = mem->n_insert;
+    out->kernel_launches = mem->launches;
+    out->candidates_filed = (int64_t)(((uint64_t)w[kDevFiledHi] << 32) | w[kDevFiledLo]);
+    out->list_cutbacks = (int64_t)w[kDevCutbacks];
+    out->longest_update_run = (int64_t)w[kDevLongestRun];
+    return EVK_OK;
 }
 
 // ---- host-buffer forms -------------------------------------------------------
@@ -519,7 +625,7 @@ int evk_select_by_value(evk_mem *mem, const int32_t *cand_ids, const int32_t *of
     if (!cand_ids || !offsets || !ids_out || !q_out) return EVK_ERR_INVALID;
     int launches = 0;
     cudaError_t err = launch_select_by_value(cand_ids, offsets, n_tasks, mem->size,
-                                             mem->q_tables + (size_t)stage * mem->cfg.capacity, k, ids_out, q_out,
+                                             mem->any_dropped ? mem->live_bits : nullptr, mem->q_tables + (size_t)stage * mem->cfg.capacity, k, ids_out, q_out,
                                              mem->status, static_cast<cudaStream_t>(stream), &launches);
     mem->launches += launches;
     return cuda_status(err);

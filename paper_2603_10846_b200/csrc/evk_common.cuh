@@ -37,6 +37,16 @@ __device__ __forceinline__ uint64_t make_key(float sim, int32_t id) {
 __device__ __forceinline__ float key_sim(uint64_t key) { return from_ordered_bits((uint32_t)(key >> 32)); }
 __device__ __forceinline__ int32_t key_id(uint64_t key) { return (int32_t)(~(uint32_t)key); }
 
+// Entries dropped from the memory: one bit per entry (1 = live) in 32-bit words.  A null pointer
+// means that nothing has ever been dropped.
+__device__ __forceinline__ bool entry_live(const uint32_t *live_bits, int64_t id) {
+    return !live_bits || ((__ldg(live_bits + (id >> 5)) >> (id & 31)) & 1u);
+}
+
+// Per-bank words in device memory (the 256-byte block at the end of the arena).
+enum DevWord { kDevStatus = 0, kDevLive = 1, kDevFiledLo = 2, kDevFiledHi = 3, kDevCutbacks = 4, kDevLongestRun = 5,
+               kDevFlag = 6, kDevDropped = 7 };
+
 // Claims one slot of a shared counter for every lane whose `want` is set, with a single atomic
 // per warp.  Every lane of the warp must call it; returns the lane's slot (undefined if !want).
 __device__ __forceinline__ int warp_claim_slot(bool want, int *counter) {

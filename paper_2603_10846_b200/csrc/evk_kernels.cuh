@@ -9,7 +9,9 @@
 namespace evk {
 
 // ---- insert (Eq. 1) ---------------------------------------------------------
-cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits, int64_t capacity,
+// live_bits: one bit per entry, set for the new entries; dev: the bank's device words (live count).
+cudaError_t launch_insert(__nv_bfloat16 *bank, float *q_tables, uint32_t *visits, uint32_t *live_bits, uint32_t *dev,
+                          int64_t capacity,
                           int d, int n_stages, int64_t first, int64_t n, const void *emb, int emb_dtype,
                           int stage, const float *q_init, float q_default, int32_t *ids_out,
                           cudaStream_t stream, int *launches);
@@ -26,6 +28,7 @@ struct StreamPlan {
     int nparts;    // thread blocks per pass (= candidate lists per query)
     int cap;       // shared-memory candidate capacity per query
     size_t smem;   // dynamic shared memory per block
+    const uint32_t *live_bits;   // entries dropped from the memory are skipped (null: none ever was)
 };
 bool stream_supported(int d);
 StreamPlan stream_plan(int64_t size, int d, int B, int k1);
@@ -47,6 +50,8 @@ struct MmaPlan {
     int n_sample;           // 0: no sampling pass
     int64_t sample_stride;  // rows between sampled entries
     int stall;              // test aid, see evk_mem_inject_stall
+    const uint32_t *live_bits;   // entries dropped from the memory are skipped (null: none ever was)
+    uint32_t *dev;               // the bank's device words (counters), or null
 };
 bool mma_supported(int d, int k1);
 MmaPlan mma_plan(int64_t size, int B, int k1);
@@ -63,8 +68,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
 constexpr int kMergeMaxParts = 2048;
 // Merges each query's lists into its pool (optionally written to pool_*_user, [B][k1]) and
 // runs phase 2 on it: ids_out / scores_out [B][k2].  norm: 0 raw mix, 1 pool z-scores.
+// live_count (may be null): device word with the number of live entries; expect is capped by it.
 cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
-                                int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                                int part_stride, int qt_size, int B, int k1, int expect, const uint32_t *live_count,
+                                int32_t *status,
                                 int32_t *pool_ids_user, float *pool_sims_user,
                                 int k2, const float *q_stage, float w, int norm, int32_t *ids_out, float *scores_out,
                                 cudaStream_t stream, int *launches);
@@ -73,9 +80,10 @@ cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_count
 size_t q_update_workspace_bytes(int64_t m);
 // visits == nullptr: constant step size alpha.  Otherwise alpha_t = 1 / visits[id] after counting
 // the update (decreasing step size), and the counts are advanced.
+// longest_run (may be null): device word raised to the longest run of one id seen in a batch.
 cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
                             int64_t m, float alpha, uint32_t *visits, int32_t *status, void *workspace,
-                            cudaStream_t stream, int *launches);
+                            cudaStream_t stream, int *launches, uint32_t *longest_run = nullptr);
 
 // Eq. 4 update with scratch held in a static device array (no caller workspace).
 int64_t q_update_static_max();
@@ -90,7 +98,7 @@ cudaError_t launch_explore(const int32_t *pool_ids, const float *pool_sims, int 
 
 // ---- start points by value (Section 3.4) -----------------------------------------------
 cudaError_t launch_select_by_value(const int32_t *cand_ids, const int32_t *offsets, int n_tasks, int64_t size,
-                                   const float *q_stage, int k, int32_t *ids_out, float *q_out, int32_t *status,
+                                   const uint32_t *live_bits, const float *q_stage, int k, int32_t *ids_out, float *q_out, int32_t *status,
                                    cudaStream_t stream, int *launches);
 
 // ---- a bank split by rows over several GPUs ---------------------------------------------
@@ -99,6 +107,17 @@ cudaError_t launch_tag_pool(const int32_t *pool_ids, int64_t n, int32_t id_offse
 cudaError_t launch_merge_shards(const int32_t *gids, const float *sims, const float *qs, int n_shards, int B, int k1,
                                 int k2, float w, int32_t *ids_out, float *scores_out, int32_t *pool_gids_out,
                                 float *pool_sims_out, cudaStream_t stream);
+
+// ---- dropping entries, export and import ---------------------------------------------------------
+// Clears the live bit of every id (the whole call is refused, through `status`, if one is out of range).
+cudaError_t launch_tombstone(const int32_t *ids, int64_t n, int64_t size, uint32_t *live_bits, uint32_t *dev,
+                             int32_t *status, cudaStream_t stream, int *launches);
+// live bits [first, first + n) as one byte per entry (1 = live).
+cudaError_t launch_live_export(const uint32_t *live_bits, int64_t first, int64_t n, uint8_t *out, cudaStream_t stream,
+                               int *launches);
+// entries [first, first + n), all live so far: those whose byte is 0 are dropped.
+cudaError_t launch_live_import(const uint8_t *live, int64_t first, int64_t n, uint32_t *live_bits, uint32_t *dev,
+                               cudaStream_t stream, int *launches);
 
 // ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
 cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);

@@ -25,7 +25,8 @@ static_assert(EVK_MAX_K1 * 3 <= kCap, "rerank scratch lives behind the pool in t
 
 __global__ void __launch_bounds__(kThreads)
 merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
-                    int part_stride, int qt_size, int k1, int expect, int32_t *__restrict__ status,
+                    int part_stride, int qt_size, int k1, int expect, const uint32_t *__restrict__ live_count,
+                    int32_t *__restrict__ status,
                     int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user,
                     int k2, const float *__restrict__ q_stage, float w, int norm,
                     int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
@@ -150,6 +151,11 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
     }
 
     int n = count;
+    // entries dropped from the memory cannot be found: the pool is as long as the live entries allow
+    if (live_count) {
+        const int live = (int)min(*live_count, (uint32_t)0x7fffffff);
+        expect = expect < live ? expect : live;
+    }
     if (n < expect && tid == 0) atomicCAS(status, 0, (int)EVK_ERR_INCOMPLETE);
     if (n > k1) {
         block_select_topk<kThreads, kSelPerThread>(keys, n, k1, hist, scal);
@@ -182,7 +188,8 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
 }  // namespace
 
 cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_counts, int nparts,
-                                int part_stride, int qt_size, int B, int k1, int expect, int32_t *status,
+                                int part_stride, int qt_size, int B, int k1, int expect, const uint32_t *live_count,
+                                int32_t *status,
                                 int32_t *pool_ids_user, float *pool_sims_user,
                                 int k2, const float *q_stage, float w, int norm, int32_t *ids_out, float *scores_out,
                                 cudaStream_t stream, int *launches) {
@@ -190,7 +197,7 @@ cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_count
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
     ++*launches;
     return launch_overlapped(merge_rerank_kernel, dim3(B), dim3(kThreads), 0, stream, part_keys, part_counts, nparts,
-                             part_stride, qt_size, k1, expect, status, pool_ids_user, pool_sims_user, k2, q_stage, w,
+                             part_stride, qt_size, k1, expect, live_count, status, pool_ids_user, pool_sims_user, k2, q_stage, w,
                              norm, ids_out, scores_out);
 }
 

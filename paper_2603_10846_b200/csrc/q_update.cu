@@ -192,7 +192,8 @@ constexpr int kLongSlots = 32;     // long runs a block can hand to its warps (m
 template <class Sorted>
 __global__ void __launch_bounds__(kApplyThreads)
 apply_runs_kernel(const Sorted sorted, int64_t m, float alpha, float *__restrict__ q_stage,
-                  uint32_t *__restrict__ visits, const int *__restrict__ flags, int32_t *__restrict__ status) {
+                  uint32_t *__restrict__ visits, const int *__restrict__ flags, int32_t *__restrict__ status,
+                  uint32_t *__restrict__ longest_run) {
     __shared__ int long_n;
     __shared__ long long long_start[kLongSlots];
     pdl_trigger();
@@ -225,6 +226,7 @@ apply_runs_kernel(const Sorted sorted, int64_t m, float alpha, float *__restrict
                     if (sorted.id(mid) == id) lo = mid; else hi = mid;
                 }
                 const int64_t end = hi;
+                if (longest_run && end - t > 8) atomicMax(longest_run, (uint32_t)(end - t));
                 if (end - t >= kLongRun) {
                     const int slot = atomicAdd(&long_n, 1);
                     if (slot < kLongSlots) {
@@ -286,7 +288,7 @@ constexpr int kSmallMax = 2048;   // above this the cluster sort is faster
 __global__ void __launch_bounds__(kSmallThreads)
 small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ rewards, int m, int n_pow2,
                     int64_t size, float alpha, float *__restrict__ q_stage, uint32_t *__restrict__ visits,
-                    int32_t *__restrict__ status) {
+                    int32_t *__restrict__ status, uint32_t *__restrict__ longest_run) {
     extern __shared__ __align__(16) unsigned char small_smem[];
     uint64_t *keys = reinterpret_cast<uint64_t *>(small_smem);        // [n_pow2] (id << 32) | position
     float *r = reinterpret_cast<float *>(keys + n_pow2);               // [m]
@@ -338,7 +340,8 @@ small_update_kernel(const int32_t *__restrict__ ids, const float *__restrict__ r
         if (t > 0 && (uint32_t)(keys[t - 1] >> 32) == id) continue;  // not the head of its run
         float q = q_stage[id];
         uint32_t seen = visits ? visits[id] : 0;
-        for (int j = t; j < m && (uint32_t)(keys[j] >> 32) == id; ++j) {
+        int j = t;
+        for (; j < m && (uint32_t)(keys[j] >> 32) == id; ++j) {
             // decreasing step size: alpha_t = 1 / (updates this entry has received, this one included)
             q = value_step(q, r[(uint32_t)keys[j]], alpha, visits != nullptr, seen);
         }
@@ -612,7 +615,7 @@ cudaError_t try_cluster_sort(const int32_t *ids, const float *rewards, int m, in
 
 cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, const float *rewards,
                             int64_t m, float alpha, uint32_t *visits, int32_t *status, void *workspace,
-                            cudaStream_t stream, int *launches) {
+                            cudaStream_t stream, int *launches, uint32_t *longest_run) {
     if (m <= 0) return cudaSuccess;
     if (m <= kSmallMax) {
         int n_pow2 = 2;
@@ -620,7 +623,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
         const size_t smem = (size_t)n_pow2 * sizeof(uint64_t) + (size_t)m * sizeof(float);
         ++*launches;
         return launch_overlapped(small_update_kernel, dim3(1), dim3(kSmallThreads), smem, stream, ids, rewards, (int)m,
-                                 n_pow2, size, alpha, q_stage, visits, status);
+                                 n_pow2, size, alpha, q_stage, visits, status, longest_run);
     }
     int bits = 0;
     while (bits < 31 && ((int64_t)1 << bits) < size) ++bits;
@@ -646,7 +649,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
             sorted.pairs = (passes & 1) ? pairs_a : pairs_b;
             ++*launches;
             return launch_overlapped(apply_runs_kernel<SortedPairs>, dim3(apply_grid), dim3(kApplyThreads), 0, stream,
-                                     sorted, m, alpha, q_stage, visits, (const int *)flags, status);
+                                     sorted, m, alpha, q_stage, visits, (const int *)flags, status, longest_run);
         }
     }
 
@@ -677,7 +680,7 @@ cudaError_t launch_q_update(float *q_stage, int64_t size, const int32_t *ids, co
     SortedArrays sorted;
     sorted.ids = k_in;
     sorted.rewards = v_in;
-    apply_runs_kernel<SortedArrays><<<apply_grid, kApplyThreads, 0, stream>>>(sorted, m, alpha, q_stage, visits, flags, status);
+    apply_runs_kernel<SortedArrays><<<apply_grid, kApplyThreads, 0, stream>>>(sorted, m, alpha, q_stage, visits, flags, status, longest_run);
     ++*launches;
     return cudaGetLastError();
 }

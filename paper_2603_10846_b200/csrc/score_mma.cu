@@ -122,6 +122,8 @@ struct MmaParams {
     int b3d;            // 1: bank stages are kSubRows rows x kSubSlices slices (contiguous bytes per row), see make_map3
     int abs_hist;       // 1: no sampled thresholds; the shared histogram bins by the similarity's own bits (see kAbsShift)
     int *anchor;        // [B] abs_hist: lowest bin of each query's histogram window + 1, 0 until the first block sets it
+    const uint32_t *live_bits;   // entries dropped from the memory are skipped (null: none ever was)
+    uint32_t *dev;      // the bank's device words: candidates filed and list cut-backs are counted there (or null)
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -703,7 +705,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             uint64_t *my_buf = p.cand + ((size_t)list_job * kBlockM + (row < 0 ? 0 : row)) * kMmaCandCap;
             // Files one similarity that reached tau_sim.
             auto file = [&](float s, int64_t row) {
-                if (row < p.size) {
+                if (row < p.size && entry_live(p.live_bits, row)) {
                     const uint64_t key = make_key(s, (int32_t)row);
                     int bin = 0;
                     if (my_hist) {
@@ -769,6 +771,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     __syncwarp();
                     const uint64_t kth = warp_select_topk(buf, n, p.k1);
                     if (lane == owner) {
+                        if (p.dev) atomicAdd(p.dev + kDevCutbacks, 1u);
                         cnt = p.k1;
                         tau_key = kth;
                         key_sim_floor = key_sim(kth);
@@ -865,7 +868,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         while (pass) {
                             const int j = __ffs(pass) - 1;
                             pass &= pass - 1;
-                            if (anchored && row0 + c0 + j < p.size) {
+                            if (anchored && row0 + c0 + j < p.size && entry_live(p.live_bits, row0 + c0 + j)) {
                                 int bin = (int)(ordered_bits(__uint_as_float(pick(va, j)) + 0.0f) >> kAbsShift) - a_base;
                                 bin = bin > kHistBins - 1 ? kHistBins - 1 : bin;
                                 atomicAdd(my_hist + bin, 1u);
@@ -929,6 +932,12 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (!real) break;
             }
             if (p.mode == 0 && ok && qt < p.n_qt && row >= 0) p.cand_cnt[(size_t)list_job * kBlockM + row] = cnt;
+            if (p.mode == 0 && p.dev) {
+                // candidates this warp leaves behind for the merge (one atomic per warp and job)
+                const unsigned left = __reduce_add_sync(0xffffffffu, (unsigned)((ok && q_valid) ? cnt : 0));
+                if (lane == 0 && left)
+                    atomicAdd(reinterpret_cast<unsigned long long *>(p.dev + kDevFiledLo), (unsigned long long)left);
+            }
         }
         slot_q[m] = -1;
         if (!ok && p.mode == 0) {
@@ -1054,7 +1063,8 @@ constexpr int kSelBins = 1024;
 
 __global__ void __launch_bounds__(kSelThreads)
 sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0,
-                        float2 *__restrict__ range, unsigned *__restrict__ hist_out) {
+                        float2 *__restrict__ range, unsigned *__restrict__ hist_out,
+                        const uint32_t *__restrict__ live_bits, int64_t sample_stride) {
     __shared__ int bins[kSelBins];
     __shared__ float red_lo[kSelThreads / 32], red_hi[kSelThreads / 32];
     __shared__ int red_cnt[kSelThreads / 32];
@@ -1072,7 +1082,9 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
     for (int j = 0; j < kSelPerThread; ++j) {
         const int i = tid + j * kSelThreads;
         float x = (i < n_sample) ? dense[(size_t)q * ld + i] : -INFINITY;
-        if (i < n_sample && !(fabsf(x) <= 3.0e38f)) x = -3.0e38f;
+        // a non-finite similarity, or a sampled entry that has been dropped from the memory, counts as
+        // the lowest value: it cannot vouch for a threshold
+        if (i < n_sample && (!(fabsf(x) <= 3.0e38f) || !entry_live(live_bits, (int64_t)i * sample_stride))) x = -3.0e38f;
         v[j] = x;
         if (i < n_sample) {
             lo = fminf(lo, x);
@@ -1342,6 +1354,8 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     pl.n_sample = (pl.pair && size >= 4 * (int64_t)kMmaSample && k1 < kMmaSample) ? kMmaSample : 0;
     pl.sample_stride = pl.n_sample ? size / pl.n_sample : 0;
     pl.stall = 0;
+    pl.live_bits = nullptr;
+    pl.dev = nullptr;
     return pl;
 }
 
@@ -1380,6 +1394,8 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.tau0 = nullptr;
     p.range = range;
     p.hist = hist;
+    p.live_bits = pl.live_bits;
+    p.dev = pl.dev;
     p.abs_hist = pl.pair ? 0 : 1;
     p.anchor = reinterpret_cast<int *>(tau0);   // the sampled thresholds' array, unused by such a scan
     // One query tile: the scan runs at HBM speed, a bank tile arrives every ~11 us and the epilogue
@@ -1425,7 +1441,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             err = cudaLaunchKernelEx(&cfg, sample_threshold_kernel, (const float *)dense, (int)kMmaSample,
-                                     (int)pl.n_sample, (int)k1, tau0, range, hist);
+                                     (int)pl.n_sample, (int)k1, tau0, range, hist, pl.live_bits, (int64_t)pl.sample_stride);
         }
         if (err != cudaSuccess) return err;
         ++*launches;

@@ -44,7 +44,8 @@ template <int QB, int NCH>
 __global__ void __launch_bounds__(kThreads)
 score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
                     const __nv_bfloat16 *__restrict__ queries, int q_base, int nq, int k1, int cap,
-                    int nparts, uint64_t *__restrict__ part_keys, int *__restrict__ part_counts) {
+                    int nparts, uint64_t *__restrict__ part_keys, int *__restrict__ part_counts,
+                    const uint32_t *__restrict__ live_bits) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t *keys = reinterpret_cast<uint64_t *>(smem_raw);          // [QB][cap]
     uint64_t *scal = keys + (size_t)QB * cap;                         // [4]
@@ -134,7 +135,7 @@ score_stream_kernel(const __nv_bfloat16 *__restrict__ bank, int64_t size, int d,
 #pragma unroll
                 for (int q = 1; q < QB; ++q)
                     if (lane == q) s = acc[r][q];
-                if (lane < nq && row < size && s >= tau_sim[lane]) {
+                if (lane < nq && row < size && s >= tau_sim[lane] && entry_live(live_bits, row)) {
                     const uint64_t key = make_key(s, (int32_t)row);
                     if (key > tau_key[lane]) {
                         const int slot = atomicAdd(&counts[lane], 1);
@@ -192,7 +193,7 @@ cudaError_t launch_one(const __nv_bfloat16 *bank, int64_t size, int d, const __n
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     kern<<<plan.nparts, kThreads, smem, stream>>>(bank, size, d, queries, q_base, nq, k1, plan.cap,
-                                                  plan.nparts, part_keys, part_counts);
+                                                  plan.nparts, part_keys, part_counts, plan.live_bits);
     return cudaGetLastError();
 }
 
@@ -255,6 +256,7 @@ bool stream_supported(int d) { return d > 0 && d % 8 == 0 && nch_for(d) != 0; }
 
 StreamPlan stream_plan(int64_t size, int d, int B, int k1) {
     StreamPlan p;
+    p.live_bits = nullptr;
     const int nch = nch_for(d);
     const int qb_max = (nch <= 4) ? 4 : 2;
     p.qb = B >= 4 ? 4 : (B >= 2 ? 2 : 1);

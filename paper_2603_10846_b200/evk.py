@@ -47,7 +47,7 @@ EXPORTS = (
     "evk_retrieve_explore", "evk_select_by_value", "evk_retrieve_local_workspace_bytes", "evk_retrieve_local",
     "evk_merge_shards", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
-    "evk_launch_count", "evk_strerror",
+    "evk_launch_count", "evk_strerror", "evk_mem_tombstone", "evk_mem_export", "evk_mem_import", "evk_mem_stats",
 )
 
 
@@ -55,6 +55,12 @@ class EvkError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+class _Stats(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int64) for name in (
+        "entries", "live_entries", "dropped_entries", "retrieve_calls", "update_calls", "insert_calls",
+        "kernel_launches", "candidates_filed", "list_cutbacks", "longest_update_run")]
 
 
 class _Config(ctypes.Structure):
@@ -113,6 +119,10 @@ def _load() -> ctypes.CDLL:
         "evk_last_status": (cint, [vp, vp]),
         "evk_launch_count": (i64, [vp]),
         "evk_strerror": (ctypes.c_char_p, [cint]),
+        "evk_mem_tombstone": (cint, [vp, vp, i64, vp]),
+        "evk_mem_export": (cint, [vp, i64, i64, vp, vp, vp, vp, vp]),
+        "evk_mem_import": (cint, [vp, i64, vp, vp, vp, vp, vp, vp]),
+        "evk_mem_stats": (cint, [vp, ctypes.POINTER(_Stats), vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -324,6 +334,51 @@ def evk_bank_read(mem: EvkMem, first: int = 0, n: Optional[int] = None, stream=N
     out = torch.empty((n, mem.d), dtype=torch.bfloat16, device=mem.arena.device)
     _check(_lib.evk_bank_read(mem.handle, first, n, _dev(out), _stream_ptr(stream)), "evk_bank_read")
     return out
+
+
+def evk_mem_tombstone(mem: EvkMem, ids: torch.Tensor, stream=None) -> None:
+    """Drop the entries `ids` (int32 CUDA tensor) from the memory; the others keep their ids."""
+    _check(_lib.evk_mem_tombstone(mem.handle, _dev(ids, torch.int32, "ids"), ids.numel(), _stream_ptr(stream)),
+           "evk_mem_tombstone")
+
+
+def evk_mem_export(mem: EvkMem, first: int = 0, n: Optional[int] = None, stream=None):
+    """Entries [first, first + n) as (rows bf16 [n][d], q fp32 [S][n], visits int32 [S][n], live uint8 [n])."""
+    n = evk_mem_size(mem) - first if n is None else n
+    dev = mem.arena.device
+    rows = torch.empty((n, mem.d), dtype=torch.bfloat16, device=dev)
+    q = torch.empty((mem.n_stages, n), dtype=torch.float32, device=dev)
+    visits = torch.empty((mem.n_stages, n), dtype=torch.int32, device=dev)
+    live = torch.empty(n, dtype=torch.uint8, device=dev)
+    _check(_lib.evk_mem_export(mem.handle, first, n, _dev(rows), _dev(q), _dev(visits), _dev(live),
+                               _stream_ptr(stream)), "evk_mem_export")
+    return rows, q, visits, live
+
+
+def evk_mem_import(mem: EvkMem, rows: torch.Tensor, q: Optional[torch.Tensor] = None,
+                   visits: Optional[torch.Tensor] = None, live: Optional[torch.Tensor] = None,
+                   return_ids: bool = False, stream=None):
+    """Append entries with their per-stage values [S][n], update counts [S][n] and live marks [n]."""
+    n = rows.shape[0]
+    if rows.dim() != 2 or rows.shape[1] != mem.d:
+        raise ValueError("rows must be [n][d]")
+    for name, t in (("q", q), ("visits", visits)):
+        if t is not None and tuple(t.shape) != (mem.n_stages, n):
+            raise ValueError(f"{name} must be [n_stages][n]")
+    if live is not None and live.numel() != n:
+        raise ValueError("live must have n elements")
+    ids = torch.empty(n, dtype=torch.int32, device=rows.device) if return_ids else None
+    _check(_lib.evk_mem_import(mem.handle, n, _dev(rows, torch.bfloat16, "rows"), _dev(q, torch.float32, "q"),
+                               _dev(visits, torch.int32, "visits"), _dev(live, torch.uint8, "live"), _dev(ids),
+                               _stream_ptr(stream)), "evk_mem_import")
+    return ids
+
+
+def evk_mem_stats(mem: EvkMem, stream=None) -> dict:
+    """Counters of the bank (synchronises the stream): see evk_stats in the header."""
+    st = _Stats()
+    _check(_lib.evk_mem_stats(mem.handle, ctypes.byref(st), _stream_ptr(stream)), "evk_mem_stats")
+    return {name: int(getattr(st, name)) for name, _ in _Stats._fields_}
 
 
 def evk_retrieve_host(mem: EvkMem, queries_host: torch.Tensor, stage: int, k1: int, k2: int, w: float,

@@ -34,14 +34,15 @@ def tol(score, scale=1.0):
     return REL * np.abs(score) + ABS * scale
 
 
-def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0, sims=None):
+def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0, sims=None, live=None):
     """Phase 1 of one query.  Returns True if the id set equals the oracle's exactly.
-    sims: this query's oracle similarities if the caller already has them."""
+    sims: this query's oracle similarities if the caller already has them; live: uint8 per entry,
+    0 for entries dropped from the memory."""
     size = bank_bits.shape[0]
-    n_pool = min(k1, size)
+    n_pool = min(k1, size if live is None else int(np.count_nonzero(live)))
     if sims is None:
         sims = oracle.sims(bank_bits, query_bits) if size else np.zeros(0)
-    o_ids, o_sims = oracle.rank(sims, k1)
+    o_ids, o_sims = oracle.rank(sims, k1, live)
     pool_ids = np.asarray(pool_ids)
     pool_sims = np.asarray(pool_sims, dtype=np.float64)
     # shape of the answer: n_pool real entries, then padding
@@ -49,6 +50,7 @@ def check_pool(bank_bits, query_bits, k1, pool_ids, pool_sims, norm_scale=1.0, s
     assert np.all(pool_ids[n_pool:] == -1) and np.all(np.isneginf(pool_sims[n_pool:])), "bad padding"
     real = pool_ids[:n_pool]
     assert len(set(real.tolist())) == n_pool, "duplicate ids in pool"
+    assert live is None or np.all(live[real] != 0), "a dropped entry is in the pool"
     if n_pool == 0:
         return True
     # similarities of the returned ids
@@ -104,7 +106,7 @@ def check_final(bank_bits, query_bits, q_stage, w, k2, pool_ids, ids, scores, no
 
 
 def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None, norm_scale=1.0, zscore=False,
-                   workers=4):
+                   workers=4, live=None):
     """out = (ids, scores, pool_ids, pool_sims) as host arrays; sample = query indices to judge.
     Returns the share of judged queries whose pool, and whose result, equal the oracle's exactly.
     Each judged query costs the oracle one scan of the bank and one full sort; `workers` queries are
@@ -116,7 +118,8 @@ def check_retrieve(bank_bits, queries_bits, q_stage, k1, k2, w, out, sample=None
 
     def judge(i):
         sims = oracle.sims(bank_bits, queries_bits[i]) if size else np.zeros(0)
-        ep = bool(check_pool(bank_bits, queries_bits[i], k1, pool_ids[i], pool_sims[i], norm_scale, sims=sims))
+        ep = bool(check_pool(bank_bits, queries_bits[i], k1, pool_ids[i], pool_sims[i], norm_scale, sims=sims,
+                             live=live))
         ef = bool(check_final(bank_bits, queries_bits[i], q_stage, w, k2, pool_ids[i], ids[i], scores[i],
                               norm_scale, zscore, sims=sims))
         return ep, ef
