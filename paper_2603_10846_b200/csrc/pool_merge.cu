@@ -17,12 +17,13 @@ namespace evk {
 
 namespace {
 
-constexpr int kThreads = 512;
+// Two shapes of the same kernel.  Few queries: 512 threads and room for 4,096 keys per query, so that
+// one query's merge is as parallel as it can be.  Hundreds of queries and pools of at most 256: blocks
+// of 128 threads with a quarter of the buffers, sixteen of which fit on an SM, so that all queries are
+// merged in one wave (1,024 queries over the clustered bank: 53 -> about 25 us).
 constexpr int kSelPerThread = 8;
-constexpr int kCap = kThreads * kSelPerThread;  // 4096 keys = 32 KB
-constexpr int kBatch = 2048;                    // candidates examined between capacity checks
-static_assert(EVK_MAX_K1 * 3 <= kCap, "rerank scratch lives behind the pool in the key buffer");
 
+template <int kThreads, int kMaxParts>
 __global__ void __launch_bounds__(kThreads)
 merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restrict__ part_counts, int nparts,
                     int part_stride, int qt_size, int k1, int expect, const uint32_t *__restrict__ live_count,
@@ -30,8 +31,11 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
                     int32_t *__restrict__ pool_ids_user, float *__restrict__ pool_sims_user,
                     int k2, const float *__restrict__ q_stage, float w, int norm,
                     int32_t *__restrict__ ids_out, float *__restrict__ scores_out) {
+    constexpr int kCap = kThreads * kSelPerThread;   // keys held at once (4,096 = 32 KB, or 1,024)
+    constexpr int kBatch = kCap / 2;                 // candidates examined between capacity checks
+    constexpr int kPoolMax = kCap / 4;               // largest pool; the rerank's scratch lives behind it
     __shared__ __align__(16) uint64_t keys[kCap];
-    __shared__ int offs[kMergeMaxParts + 1];
+    __shared__ int offs[kMaxParts + 1];
     __shared__ int hist[256];
     __shared__ uint64_t scal[4];
     __shared__ int count;
@@ -180,8 +184,8 @@ merge_rerank_kernel(const uint64_t *__restrict__ part_keys, const int *__restric
     }
     __syncthreads();
     // phase 2 on the pool keys[0..n) (any order); scratch behind the pool
-    uint64_t *skey = keys + EVK_MAX_K1;
-    int32_t *sid = reinterpret_cast<int32_t *>(keys + 2 * EVK_MAX_K1);
+    uint64_t *skey = keys + kPoolMax;
+    int32_t *sid = reinterpret_cast<int32_t *>(keys + 2 * kPoolMax);
     rerank_block<kThreads>(keys, n, k2, q_stage, w, norm, skey, sid, ids_out + (size_t)q * k2, scores_out + (size_t)q * k2);
 }
 
@@ -193,12 +197,17 @@ cudaError_t launch_merge_rerank(const uint64_t *part_keys, const int *part_count
                                 int32_t *pool_ids_user, float *pool_sims_user,
                                 int k2, const float *q_stage, float w, int norm, int32_t *ids_out, float *scores_out,
                                 cudaStream_t stream, int *launches) {
+    static_assert(EVK_MAX_K1 * 4 <= 512 * kSelPerThread, "the large shape holds the largest pool");
     if (B <= 0) return cudaSuccess;
     if (nparts > kMergeMaxParts) return cudaErrorInvalidValue;
     ++*launches;
-    return launch_overlapped(merge_rerank_kernel, dim3(B), dim3(kThreads), 0, stream, part_keys, part_counts, nparts,
-                             part_stride, qt_size, k1, expect, live_count, status, pool_ids_user, pool_sims_user, k2, q_stage, w,
-                             norm, ids_out, scores_out);
+    if (B >= 256 && k1 <= 256 && nparts <= 255)
+        return launch_overlapped(merge_rerank_kernel<128, 255>, dim3(B), dim3(128), 0, stream, part_keys, part_counts,
+                                 nparts, part_stride, qt_size, k1, expect, live_count, status, pool_ids_user,
+                                 pool_sims_user, k2, q_stage, w, norm, ids_out, scores_out);
+    return launch_overlapped(merge_rerank_kernel<512, kMergeMaxParts>, dim3(B), dim3(512), 0, stream, part_keys,
+                             part_counts, nparts, part_stride, qt_size, k1, expect, live_count, status, pool_ids_user,
+                             pool_sims_user, k2, q_stage, w, norm, ids_out, scores_out);
 }
 
 }  // namespace evk
