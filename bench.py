@@ -282,6 +282,12 @@ class Bank:
         return query_sets, r_sets, own_updates
 
 
+def check_status(evk, mem):
+    st = evk.evk_last_status(mem)
+    if st != 0:
+        raise RuntimeError(f"device status {st}: {evk.strerror(st)}")
+
+
 def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 0.0, parts=("device",),
             sample_clocks=True, peaks=None):
     """Times one configuration on a resident bank.  steps > 0: exactly that many timed steps;
@@ -358,7 +364,7 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         for i in range(max(warmup, 3)):
             step(i, 1 if bk.n_local >= 1024 else 0)
         torch.cuda.synchronize()
-        assert evk.evk_last_status(mem) == 0
+        check_status(evk, mem)
         # a short probe sizes a time-based leg
         a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
@@ -390,7 +396,7 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         sync_all()
         clocks = sampler.stop() if (rank == 0 and sample_clocks) else None
         elapsed_ms = max_over_ranks(t_start.elapsed_time(t_stop))
-        assert evk.evk_last_status(mem) == 0
+        check_status(evk, mem)
         size_end = evk.evk_mem_size(mem)
         rows = 0.5 * (size_start + size_end)
         res.update({"steps": k, "ms_per_step": elapsed_ms / k, "elapsed_ms": elapsed_ms,
@@ -445,7 +451,7 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         c.record(stream)
         torch.cuda.synchronize()
         us = 1e3 * a.elapsed_time(c) / iters
-        assert evk.evk_last_status(mem) == 0
+        check_status(evk, mem)
         res["update_only"] = {"us_per_batch": us, "updates": int(n_upd), "iters": iters,
                               "updates_per_s": n_upd / (us * 1e-6) if us > 0 else None,
                               "longest_duplicate_chain": longest}
@@ -481,7 +487,7 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         c.record(stream)
         sync_all()
         e2e_ms = max_over_ranks(a.elapsed_time(c))
-        assert evk.evk_last_status(mem) == 0
+        check_status(evk, mem)
         res["e2e"] = {"value": world * b * k / (e2e_ms * 1e-3), "unit": UNIT,
                       "h2d_bytes_per_step": n_new * wl.d * 2 + b * wl.d * 2 + n_upd * 8,
                       "d2h_bytes_per_step": b * wl.k2 * 8, "ms_per_step": e2e_ms / k, "steps": k,

@@ -600,15 +600,16 @@ cudaError_t try_cluster_sort(const int32_t *ids, const float *rewards, int m, in
     cfg.blockDim = dim3(kClThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    // A plain launch, not a programmatic dependent one: on B200 (driver 580) a kernel launched as a
+    // cluster with that attribute was seen to run past its griddepcontrol.wait while the kernel before
+    // it (the merge that writes the ids) was still running.
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = NB;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = 1;
     *launched = true;
     return cudaLaunchKernelEx(&cfg, kern, ids, rewards, m, size, flags, pairs_a, pairs_b, passes);
 }

@@ -1482,7 +1482,10 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     if (ev_start) err = cudaEventRecord(ev_start, stream);
     // behind the threshold (or reset) kernel the scan may start early; its epilogue waits for that kernel
     if (err == cudaSuccess)
-        err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, (pl.n_sample != 0 || p.abs_hist) && !ev_start,
+        // (Only a scan of single blocks starts early.  A kernel launched as a cluster with the programmatic
+        // attribute was seen, on B200 with driver 580, to run past its griddepcontrol.wait while its
+        // predecessor was still running, so the paired scan is launched in plain stream order.)
+        err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, p.abs_hist && !pl.pair && !ev_start,
                             pl.pair != 0, stream);
     if (err != cudaSuccess) return err;
     ++*launches;

@@ -484,6 +484,38 @@ def test_host_buffer_entry_points(evk):
     parity.check_update(q_tab[0], ids.numpy(), r.numpy(), 0.25, evk.evk_q_read(mem, 0).cpu().numpy())
 
 
+@pytest.mark.parametrize("b,k2", [(64, 16), (300, 8), (2100, 32)])
+def test_kernels_of_one_stream_wait_for_one_another(evk, b, k2):
+    """The kernels of a retrieval and of the update behind it are chained so that one may start while
+    its predecessor still runs; each must wait before it reads what the predecessor writes.  Buffers
+    are filled with garbage first, so that a kernel that ran ahead would read garbage: the scratch of
+    the retrieval (stale thresholds, counters and candidate lists) and the result ids that the update
+    consumes (1,024 ids: the single-block update; 2,400: the one-cluster sort; 67,200: the
+    multi-launch sort)."""
+    n, d, k1 = 50000, 64, 64
+    bank = synth.gaussian_unit(n, d, 401, DEV)
+    q_tab = np.random.default_rng(402).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    queries = [synth.gaussian_unit(b, d, 403 + j, DEV) for j in range(3)]
+    clean = []
+    for qs in queries:
+        clean.append(evk.evk_retrieve(mem, qs, 0, k1, k2, 0.5)[0].clone())
+        torch.cuda.synchronize()
+    ids = torch.empty((b, k2), dtype=torch.int32, device=DEV)
+    scores = torch.empty((b, k2), dtype=torch.float32, device=DEV)
+    rewards = torch.from_numpy(np.random.default_rng(404).random(b * k2).astype(np.float32)).to(DEV)
+    q_orc = q_tab[1].copy()
+    for it in range(12):
+        ids.fill_(0x7f7f7f7f)
+        mem._ws["retrieve"].fill_(0x7f)
+        evk.evk_retrieve(mem, queries[it % 3], 0, k1, k2, 0.5, out=(ids, scores))
+        evk.evk_q_update(mem, ids.reshape(-1), 1, rewards, 0.2)
+        assert evk.evk_last_status(mem) == 0, it
+        assert torch.equal(ids, clean[it % 3]), it
+        q_orc = oracle.q_update_f32(q_orc, ids.reshape(-1).cpu().numpy(), rewards.cpu().numpy(), 0.2)
+    assert np.array_equal(evk.evk_q_read(mem, 1).cpu().numpy().view(np.uint32), q_orc.view(np.uint32))
+
+
 def test_host_buffer_calls_check_arguments_before_copying(evk):
     # a refused call enqueues nothing: no kernel is launched, the outputs keep their contents
     n, d, b, k1, k2 = 5000, 128, 4, 32, 4
