@@ -38,9 +38,9 @@ UNIT = "queries/s"
 NOMINAL_HBM_GBS = 8000.0          # the HBM3e figure the bandwidth target is quoted against
 # DRAM bytes (read + written) per scanned bank entry of width 1024, from one ncu capture of the
 # scan kernel; see TRAFFIC_SOURCE.  The bank is read once per launch, so traffic grows with the rows.
-SCAN_DRAM_BYTES_PER_ENTRY = 542.93e6 / 262224
+SCAN_DRAM_BYTES_PER_ENTRY = 541.80e6 / 262147
 TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one score_mma_kernel launch, "
-                  "262,224 rows x 1024 bf16 (512 MiB), 64 queries, k1=128: 542.93 MB = 2,070.5 B per entry "
+                  "262,147 rows x 1024 bf16 (512 MiB), 64 queries, k1=128: 537.81 + 3.99 MB = 2,066.8 B per entry "
                   "against 2,048 B algorithmic; scaled by the rows one launch scans")
 
 
@@ -227,6 +227,8 @@ def scan_roofline(evk, kind, n_score_launches, wl, b, rows, scan_ms, peaks, cloc
         "gbs": gbs, "tflops": tflops,
         "frac_of_copy_hbm": gbs / peaks["hbm_gbs"],
         "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS,
+        # against a read-only stream of the same bank through the same copy engine, measured in this run
+        "frac_of_read_only_hbm": gbs / peaks["hbm_read_gbs"] if peaks.get("hbm_read_gbs") else None,
         "frac_of_burst_tensor": tflops / peaks["bf16_tflops"],
         "frac_of_sustained_tensor": tflops / peaks["bf16_tflops_sustained"],
         # clock-normalised duration: compare legs that ran at different SM clocks
@@ -550,6 +552,28 @@ def run_evk(args):
     bk = Bank(evk, synth, parallel, wl, dev, rank, world, args.scoring, args.layout)
     rows_layout = args.layout == "rows" and world > 1
 
+    # ---- calibration: what a kernel that only reads can reach on this GPU, on this bank ----
+    read_gbs = None
+    if wl.n * wl.d * 2 > 126e6:
+        stream = torch.cuda.current_stream()
+        for _ in range(3):
+            evk.evk_mem_read_probe(bk.mem)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(20):
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            evk.evk_mem_read_probe(bk.mem)
+            c.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(c))
+        check_status(evk, bk.mem)
+        read_bytes = (evk.evk_mem_size(bk.mem) * wl.d * 2 // 32768) * 32768
+        read_gbs = {"best": read_bytes / (min(times) * 1e-3) / 1e9, "mean": read_bytes / (statistics.mean(times) * 1e-3) / 1e9,
+                    "launches": len(times), "how": "evk_mem_read_probe: the stored rows streamed once into shared memory, "
+                                                   "32 KB bulk copies, one block per SM, CUDA events around each launch"}
+        peaks["hbm_read_gbs"] = read_gbs["mean"]
+
     # ---- headline: exactly --steps steps (or about a second of them) ----
     head = run_leg(bk, b, args.warmup, steps=args.steps, min_seconds=1.0,
                    parts=("device", "retrieve", "update", "e2e"), peaks=peaks)
@@ -588,6 +612,7 @@ def run_evk(args):
             "update_only": head.get("update_only"),
             "gpu_launches": head["gpu_launches"],
             "clocks": head["clocks"],
+            "hbm_read_only": read_gbs,
             "sustained": {"steps": sustained["steps"], "seconds": sustained["elapsed_ms"] / 1e3,
                           "ms_per_step": sustained["ms_per_step"], "queries_per_s": sustained["queries_per_s"],
                           "roofline": sustained.get("roofline"), "clocks": sustained["clocks"]},

@@ -350,6 +350,12 @@ int evk_retrieve_plan(const evk_mem *mem, int32_t B, int32_t k1, int32_t *kind_o
  * setting is used by one call and then cleared; NULLs clear it. */
 int evk_mem_profile_scoring(evk_mem *mem, void *start_event, void *stop_event);
 
+/* Measurement aid (no counterpart in the paper): reads the stored rows once, 32 KB at a time, into
+ * shared memory with the copy engine the scans use, and drops them: one kernel on `stream`.  Timed
+ * by the caller, bytes = size * d * 2 over its duration is the read-only bandwidth of this GPU, the
+ * ceiling of a scan (a copy's measured bandwidth counts reads and writes and lies below it). */
+int evk_mem_read_probe(evk_mem *mem, void *stream);
+
 /* Failure-detection test aid.  The next evk_retrieve that runs the tensor kernel starves its
  * own pipeline: the producer warp issues no loads, so the consumer's bounded wait (shortened to
  * about a tenth of a second for this call) runs out.  Nothing faults or hangs: every block

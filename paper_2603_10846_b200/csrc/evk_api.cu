@@ -482,6 +482,15 @@ int evk_mem_import(evk_mem *mem, int64_t n, const void *rows_bf16, const float *
     return cuda_status(err);
 }
 
+int evk_mem_read_probe(evk_mem *mem, void *stream) {
+    if (!mem) return EVK_ERR_INVALID;
+    if (mem->size <= 0) return EVK_OK;
+    const cudaError_t err = launch_read_probe(mem->bank, (size_t)mem->size * mem->cfg.d * sizeof(__nv_bfloat16),
+                                              mem->status, static_cast<cudaStream_t>(stream));
+    ++mem->launches;
+    return cuda_status(err);
+}
+
 int evk_mem_stats(evk_mem *mem, evk_stats *out, void *stream_v) {
     if (!mem || !out) return EVK_ERR_INVALID;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);

@@ -119,6 +119,10 @@ cudaError_t launch_live_export(const uint32_t *live_bits, int64_t first, int64_t
 cudaError_t launch_live_import(const uint8_t *live, int64_t first, int64_t n, uint32_t *live_bits, uint32_t *dev,
                                cudaStream_t stream, int *launches);
 
+// ---- read-only bandwidth calibration ---------------------------------------------------------------
+// Streams `bytes` (rounded down to whole 32 KB pieces) of device memory into shared memory once.
+cudaError_t launch_read_probe(const void *src, size_t bytes, int32_t *status, cudaStream_t stream);
+
 // ---- rewards (Eq. 5, Eq. 6, running normalisation) ---------------------------------
 cudaError_t launch_reward_draft(const uint8_t *feasible, int64_t n, float *out, cudaStream_t stream);
 cudaError_t launch_reward_refine(const float *best, const float *latency, const uint8_t *feasible, int64_t n,

@@ -48,6 +48,7 @@ EXPORTS = (
     "evk_merge_shards", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
     "evk_launch_count", "evk_strerror", "evk_mem_tombstone", "evk_mem_export", "evk_mem_import", "evk_mem_stats",
+    "evk_mem_read_probe",
 )
 
 
@@ -123,6 +124,7 @@ def _load() -> ctypes.CDLL:
         "evk_mem_export": (cint, [vp, i64, i64, vp, vp, vp, vp, vp]),
         "evk_mem_import": (cint, [vp, i64, vp, vp, vp, vp, vp, vp]),
         "evk_mem_stats": (cint, [vp, ctypes.POINTER(_Stats), vp]),
+        "evk_mem_read_probe": (cint, [vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -379,6 +381,11 @@ def evk_mem_stats(mem: EvkMem, stream=None) -> dict:
     st = _Stats()
     _check(_lib.evk_mem_stats(mem.handle, ctypes.byref(st), _stream_ptr(stream)), "evk_mem_stats")
     return {name: int(getattr(st, name)) for name, _ in _Stats._fields_}
+
+
+def evk_mem_read_probe(mem: EvkMem, stream=None) -> None:
+    """Measurement aid: stream the stored rows once into shared memory (time it with CUDA events)."""
+    _check(_lib.evk_mem_read_probe(mem.handle, _stream_ptr(stream)), "evk_mem_read_probe")
 
 
 def evk_retrieve_host(mem: EvkMem, queries_host: torch.Tensor, stage: int, k1: int, k2: int, w: float,
