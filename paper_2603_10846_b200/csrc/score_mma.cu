@@ -446,7 +446,12 @@ __device__ __noinline__ uint64_t warp_select_topk(uint64_t *buf, int n, int k) {
 
 // ---- the kernel ---------------------------------------------------------------
 
-template <bool kPair>
+// kPair: clusters of two blocks on 256-query tiles.  kMode: 0 filter (the scan proper), 1 dense (every
+// similarity of a small sample is written out).  kAbs: thresholds started off by the scan itself
+// (scans of one query tile) instead of sampled ones.  Three shapes are built: <false, 0, true>,
+// <true, 0, false> and <false, 1, false>; each carries only its own code (the epilogue's speed
+// depends on how much code it has to run through).
+template <bool kPair, int kMode, bool kAbs>
 __global__ void __launch_bounds__(kThreads, 1)
 score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
                  const MmaParams p) {
@@ -491,7 +496,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         reinterpret_cast<volatile unsigned long long *>(reinterpret_cast<unsigned char *>(bars) + 256 + 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool abs_mode = p.abs_hist != 0;
+    constexpr bool abs_mode = kAbs;
     const long long wait_limit = p.stall ? kTimeoutCycles / 16 : kTimeoutCycles;
     pdl_trigger();
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
@@ -540,11 +545,11 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // ===== TMA producer =====
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
-            bool ok = !(p.stall && p.mode == 0);
+            bool ok = !(p.stall && kMode == 0);
             // one query tile (or one pair of them): every bank tile is read exactly once.  With more,
             // the blocks that share a tile read it within a few tiles of one another, and the hint
             // would let it go in between (4,096 queries over 6 GiB: 22.7 against 19.5 ms).
-            const bool stream_once = p.mode == 0 && (kPair ? p.n_qt <= 2 : p.n_qt == 1);
+            const bool stream_once = kMode == 0 && (kPair ? p.n_qt <= 2 : p.n_qt == 1);
             const uint64_t bank_policy = l2_evict_first_policy();
             if (ok && p.a_resident && worker < n_jobs) {
                 a_armed = true;
@@ -724,7 +729,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             };
             // One chunk of columns: store it (dense mode) or file the entries that pass the filters.
             auto process = [&](uint32_t (&v)[kChunk], int64_t row0, int c0) {
-                if (p.mode == 1) {
+                if (kMode == 1) {
                     if (q_valid) {
                         float4 *dst = reinterpret_cast<float4 *>(p.dense + (size_t)q * p.dense_ld + row0 + c0);
 #pragma unroll
@@ -813,7 +818,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
                 }
                 uint32_t va[kChunk], vb[kChunk];
-                if (real && abs_mode && p.mode == 0 && t == split) {
+                if (real && abs_mode && kMode == 0 && t == split) {
                     // The job's first tile starts the histogram off (every lane of the warp walks through this,
                     // the tensor-memory loads being warp-wide).  The window is anchored by whoever comes first,
                     // and the tile's entries from window bin kBootBin up are counted.  Filing waits until the
@@ -932,8 +937,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 held = false;
                 if (!real) break;
             }
-            if (p.mode == 0 && ok && qt < p.n_qt && row >= 0) p.cand_cnt[(size_t)list_job * kBlockM + row] = cnt;
-            if (p.mode == 0 && p.dev) {
+            if (kMode == 0 && ok && qt < p.n_qt && row >= 0) p.cand_cnt[(size_t)list_job * kBlockM + row] = cnt;
+            if (kMode == 0 && p.dev) {
                 // candidates this warp leaves behind for the merge (one atomic per warp and job)
                 const unsigned left = __reduce_add_sync(0xffffffffu, (unsigned)((ok && q_valid) ? cnt : 0));
                 if (lane == 0 && left)
@@ -941,7 +946,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
         slot_q[m] = -1;
-        if (!ok && p.mode == 0) {
+        if (!ok && kMode == 0) {
             // aborting: whatever this block was to deliver counts as empty, so the merge reads nothing stale
             for (int job = worker; job < n_jobs; job += n_workers) {
                 const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
@@ -958,7 +963,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // of the scan old lets through an eighth more).  Reading them after every tile throughout
         // costs a tenth of the kernel's time: the reads of all blocks meet the survivors' atomic
         // updates on the same L2 lines.
-        if (p.mode == 0 && (p.tau0 != nullptr || abs_mode) && p.sync_tiles != kSyncAlways) {
+        if (kMode == 0 && (p.tau0 != nullptr || abs_mode) && p.sync_tiles != kSyncAlways) {
             pdl_wait();
             const long long t0 = clock64();
             int seen = -1, job_start = 0, next_poll = 0, q_first = -2;
@@ -1253,7 +1258,8 @@ SmemPlan smem_plan(int B, int d) {
 // pair = true: clusters of two blocks (grid must be even), the cta_group::2 variant.
 cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
                           size_t smem_bytes, bool overlap, bool pair, cudaStream_t stream) {
-    auto kern = pair ? score_mma_kernel<true> : score_mma_kernel<false>;
+    auto kern = pair ? score_mma_kernel<true, 0, false>
+                     : (p.mode == 1 ? score_mma_kernel<false, 1, false> : score_mma_kernel<false, 0, true>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
