@@ -264,7 +264,6 @@ class Bank:
         del bank
         self.new_rows = synth.gaussian_unit(16, wl.d, 77 + rank, dev)
         self.new_rows_host = self.new_rows.cpu().pin_memory()
-        self.new_rows_stage = torch.empty_like(self.new_rows)
 
     def inputs(self, b, n_batches):
         """Query batches, per-query rewards and (for a workload with its own update stream) update batches."""
@@ -468,11 +467,12 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         k = res.get("steps") or pick_steps(1.0)
         n_new = rows_per_step(k)
 
+        evk.evk_mem_set_host_staging(mem, 8 << 20)
+
         def e2e_step(i):
             stage = i % 2
             if n_new:
-                bk.new_rows_stage[:n_new].copy_(bk.new_rows_host[:n_new], non_blocking=True)
-                evk.evk_mem_insert(mem, bk.new_rows_stage[:n_new], evk.EVK_STAGE_ALL)
+                evk.evk_mem_insert_host(mem, bk.new_rows_host[:n_new], evk.EVK_STAGE_ALL)
             evk.evk_retrieve_host(mem, q_host[i % 4], stage, wl.k1, wl.k2, wl.w, ids_h, sc_h)
             if upd_h:
                 evk.evk_q_update_host(mem, upd_h[i % len(upd_h)][0], stage, upd_h[i % len(upd_h)][1], wl.alpha)
@@ -493,7 +493,10 @@ def run_leg(bk: Bank, b: int, warmup: int, steps: int = 0, min_seconds: float = 
         res["e2e"] = {"value": world * b * k / (e2e_ms * 1e-3), "unit": UNIT,
                       "h2d_bytes_per_step": n_new * wl.d * 2 + b * wl.d * 2 + n_upd * 8,
                       "d2h_bytes_per_step": b * wl.k2 * 8, "ms_per_step": e2e_ms / k, "steps": k,
-                      "step": f"insert {n_new} rows from a pinned host buffer + evk_retrieve_host + evk_q_update_host"}
+                      "step": f"evk_mem_insert_host ({n_new} rows) + evk_retrieve_host + evk_q_update_host, all from pinned host "
+                              "arrays, through a page-locked staging buffer (evk_mem_set_host_staging): the result is read "
+                              "on the host every step"}
+        evk.evk_mem_set_host_staging(mem, 0)
     return res
 
 

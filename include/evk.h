@@ -253,11 +253,30 @@ typedef struct evk_stats {
 } evk_stats;
 int evk_mem_stats(evk_mem *mem, evk_stats *out, void *stream);
 
-/* Host-buffer forms of the two hot calls, for callers whose data lives in host
- * memory (pinned memory makes the copies asynchronous).  They copy the inputs to
- * the device, run the same kernels, copy the results back and synchronise the
- * stream before returning.  `workspace` must hold the *_host_workspace_bytes
- * amount (device memory: staging plus the kernel workspace). */
+/* Host-buffer forms of the three hot calls, for callers whose data lives in host memory (the
+ * loop of Section 3.2 is driven from the host: queries, rewards and new entries arrive there).
+ * They copy the inputs to the device and run the same kernels.  Every host-side check of the
+ * device-pointer form is made before anything is copied.  `workspace` is DEVICE memory of the
+ * *_host_workspace_bytes amount (staging plus the kernel workspace), 256-byte aligned.
+ *
+ * Without a staging buffer each call synchronises the stream before it returns (the caller's
+ * arrays may be pageable; they are the caller's again on return whatever the outcome).
+ *
+ * evk_mem_set_host_staging hands the library a page-locked, device-visible host buffer
+ * (cudaHostAlloc / cudaHostRegister memory; 256-byte aligned, at least 16 KB; it stays the
+ * caller's and must outlive the handle or be withdrawn with pinned_host = NULL, which waits for
+ * the work that still reads it).  It is cut into four slots used in turn.  Then, for inputs that
+ * fit one slot:
+ *   - evk_q_update_host and evk_mem_insert_host copy the caller's arrays into a slot (host
+ *     memcpy), enqueue the transfer and the kernels, and return WITHOUT waiting for the device:
+ *     the caller's arrays are free on return, and what the device finds (an id out of range)
+ *     reaches the status word exactly as with evk_q_update;
+ *   - evk_retrieve_host lets the merge kernel write ids and scores straight into a slot, waits
+ *     for the stream, and copies them to ids_out_host / scores_out_host.
+ * Larger inputs take the path without staging.  EVK_ERR_INVALID if the buffer is not page-locked
+ * host memory the device can address.  evk_mem_insert_host assigns ids like evk_mem_insert (the
+ * next n ids in row order) and does not return them. */
+int evk_mem_set_host_staging(evk_mem *mem, void *pinned_host, size_t bytes);
 size_t evk_retrieve_host_workspace_bytes(const evk_mem *mem, int32_t B, int32_t k1, int32_t k2);
 int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32_t B, int stage,
                       int32_t k1, int32_t k2, float w,
@@ -267,6 +286,9 @@ size_t evk_q_update_host_workspace_bytes(const evk_mem *mem, int64_t M);
 int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stage,
                       const float *rewards_host, float alpha,
                       void *workspace, size_t workspace_bytes, void *stream);
+size_t evk_mem_insert_host_workspace_bytes(const evk_mem *mem, int64_t n);
+int evk_mem_insert_host(evk_mem *mem, const void *emb_host, int emb_dtype, int64_t n, int stage,
+                        const float *q_init_host, void *workspace, size_t workspace_bytes, void *stream);
 
 /* evk_retrieve with epsilon-greedy exploration (Section 3.3: the context is drawn from the
  * pool with an epsilon-greedy policy over the stage's values).  Per query, word 0 of a

@@ -45,6 +45,14 @@ struct evk_mem {
     int stall_next;       // evk_mem_inject_stall: the next tensor-path retrieve starves its consumer
     int64_t launches;
     cudaEvent_t prof_start, prof_stop;  // armed by evk_mem_profile_scoring for one retrieve
+    // the caller's page-locked staging buffer (evk_mem_set_host_staging), cut into slots used in turn;
+    // a slot's event marks the end of the device work that reads it
+    char *stage_host;     // host address of slot 0, nullptr = none
+    char *stage_dev;      // the same memory as the device sees it
+    size_t slot_bytes;
+    int slot_next;
+    bool slot_busy[4];
+    cudaEvent_t slot_ev[4];
 };
 
 namespace {
@@ -118,6 +126,37 @@ bool stage_ok(const evk_mem *m, int stage) { return stage >= 0 && stage < m->cfg
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? EVK_OK : EVK_ERR_CUDA; }
 
+constexpr int kHostSlots = 4;
+
+// The next staging slot, once the device work that read it last has ended.  -1 if that wait fails.
+int acquire_slot(evk_mem *m) {
+    const int s = m->slot_next;
+    m->slot_next = (s + 1) % kHostSlots;
+    if (m->slot_busy[s]) {
+        if (cudaEventSynchronize(m->slot_ev[s]) != cudaSuccess) return -1;
+        m->slot_busy[s] = false;
+    }
+    return s;
+}
+
+// Marks the slot as read by everything enqueued on `stream` so far.
+bool release_slot_after(evk_mem *m, int s, cudaStream_t stream) {
+    if (cudaEventRecord(m->slot_ev[s], stream) != cudaSuccess) return false;
+    m->slot_busy[s] = true;
+    return true;
+}
+
+void drop_staging(evk_mem *m) {
+    if (!m->stage_host) return;
+    for (int s = 0; s < kHostSlots; ++s) {
+        if (m->slot_busy[s]) (void)cudaEventSynchronize(m->slot_ev[s]);
+        (void)cudaEventDestroy(m->slot_ev[s]);
+        m->slot_busy[s] = false;
+    }
+    m->stage_host = m->stage_dev = nullptr;
+    m->slot_bytes = 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -151,6 +190,10 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
     m->stall_next = 0;
     m->launches = 0;
     m->prof_start = m->prof_stop = nullptr;
+    m->stage_host = m->stage_dev = nullptr;
+    m->slot_bytes = 0;
+    m->slot_next = 0;
+    for (int s = 0; s < kHostSlots; ++s) m->slot_busy[s] = false;
     cudaError_t err = cudaMemsetAsync(m->status, 0, 256, 0);
     if (err == cudaSuccess) err = cudaStreamSynchronize(0);
     if (err != cudaSuccess) {
@@ -162,7 +205,36 @@ int evk_mem_create(const evk_config *cfg, evk_mem **out) {
 }
 
 int evk_mem_destroy(evk_mem *mem) {
+    if (mem) drop_staging(mem);
     delete mem;
+    return EVK_OK;
+}
+
+int evk_mem_set_host_staging(evk_mem *mem, void *pinned_host, size_t bytes) {
+    if (!mem) return EVK_ERR_INVALID;
+    if (!pinned_host) {
+        drop_staging(mem);
+        return EVK_OK;
+    }
+    if (!aligned(pinned_host, 256) || bytes / kHostSlots < 4096) return EVK_ERR_INVALID;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, pinned_host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return EVK_ERR_INVALID;
+    }
+    // page-locked and visible to the device: the result of a retrieval is written straight into it
+    if (attr.type != cudaMemoryTypeHost || !attr.devicePointer) return EVK_ERR_INVALID;
+    drop_staging(mem);
+    for (int s = 0; s < kHostSlots; ++s) {
+        if (cudaEventCreateWithFlags(&mem->slot_ev[s], cudaEventDisableTiming) != cudaSuccess) {
+            for (int t = 0; t < s; ++t) (void)cudaEventDestroy(mem->slot_ev[t]);
+            return EVK_ERR_CUDA;
+        }
+    }
+    mem->stage_host = static_cast<char *>(pinned_host);
+    mem->stage_dev = static_cast<char *>(attr.devicePointer);
+    mem->slot_bytes = (bytes / kHostSlots) & ~(size_t)255;
+    mem->slot_next = 0;
     return EVK_OK;
 }
 
@@ -543,18 +615,39 @@ int evk_retrieve_host(evk_mem *mem, const void *queries_host, int q_dtype, int32
     float *scores_dev = reinterpret_cast<float *>(reinterpret_cast<char *>(ids_dev) + align256(b * k2 * sizeof(float)));
     char *inner = reinterpret_cast<char *>(scores_dev) + align256(b * k2 * sizeof(float));
     const size_t inner_bytes = workspace_bytes - (size_t)(inner - ws);
+    // with a staging buffer the result is written into it by the merge kernel itself and handed over
+    // after the synchronise; without one it is copied back from the workspace
+    const size_t res_bytes = align256(b * k2 * sizeof(int32_t)) + b * k2 * sizeof(float);
+    int slot = -1;
+    if (mem->stage_host && res_bytes <= mem->slot_bytes) {
+        slot = acquire_slot(mem);
+        if (slot < 0) return EVK_ERR_CUDA;
+    }
     if (cudaMemcpyAsync(q_dev, queries_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return EVK_ERR_CUDA;
     // from here on a copy may be in flight: every return synchronises, so that the caller's host
     // buffers are its own again whatever the outcome
-    int rc = evk_retrieve(mem, q_dev, q_dtype, B, stage, k1, k2, w, ids_dev, scores_dev, nullptr, nullptr,
+    int rc;
+    if (slot >= 0) {
+        char *res_dev = mem->stage_dev + (size_t)slot * mem->slot_bytes;
+        rc = evk_retrieve(mem, q_dev, q_dtype, B, stage, k1, k2, w, reinterpret_cast<int32_t *>(res_dev),
+                          reinterpret_cast<float *>(res_dev + align256(b * k2 * sizeof(int32_t))), nullptr, nullptr,
                           inner, inner_bytes, stream_v);
-    if (rc == EVK_OK &&
-        (cudaMemcpyAsync(ids_out_host, ids_dev, b * k2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-         cudaMemcpyAsync(scores_out_host, scores_dev, b * k2 * sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess))
-        rc = EVK_ERR_CUDA;
+    } else {
+        rc = evk_retrieve(mem, q_dev, q_dtype, B, stage, k1, k2, w, ids_dev, scores_dev, nullptr, nullptr,
+                          inner, inner_bytes, stream_v);
+        if (rc == EVK_OK &&
+            (cudaMemcpyAsync(ids_out_host, ids_dev, b * k2 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+             cudaMemcpyAsync(scores_out_host, scores_dev, b * k2 * sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess))
+            rc = EVK_ERR_CUDA;
+    }
     const cudaError_t sync = cudaStreamSynchronize(stream);
     if (rc == EVK_OK && sync != cudaSuccess) rc = EVK_ERR_CUDA;
+    if (rc == EVK_OK && slot >= 0) {
+        const char *res = mem->stage_host + (size_t)slot * mem->slot_bytes;
+        memcpy(ids_out_host, res, b * k2 * sizeof(int32_t));
+        memcpy(scores_out_host, res + align256(b * k2 * sizeof(int32_t)), b * k2 * sizeof(float));
+    }
     return rc;
 }
 
@@ -578,6 +671,23 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
     int32_t *ids_dev = reinterpret_cast<int32_t *>(ws);
     float *r_dev = reinterpret_cast<float *>(ws + align256((size_t)M * 4));
     char *inner = ws + 2 * align256((size_t)M * 4);
+    const size_t r_off = align256((size_t)M * 4);
+    if (mem->stage_host && r_off + (size_t)M * 4 <= mem->slot_bytes) {
+        // staged: the batch is copied into the page-locked slot here and travels from there, so the
+        // caller's arrays are its own again on return and nothing waits for the device
+        const int slot = acquire_slot(mem);
+        if (slot < 0) return EVK_ERR_CUDA;
+        char *h = mem->stage_host + (size_t)slot * mem->slot_bytes;
+        memcpy(h, ids_host, (size_t)M * 4);
+        memcpy(h + r_off, rewards_host, (size_t)M * 4);
+        if (cudaMemcpyAsync(ids_dev, h, r_off + (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return EVK_ERR_CUDA;
+        if (!release_slot_after(mem, slot, stream)) {
+            (void)cudaStreamSynchronize(stream);
+            return EVK_ERR_CUDA;
+        }
+        return evk_q_update(mem, ids_dev, M, stage, r_dev, alpha, inner, workspace_bytes - (size_t)(inner - ws), stream_v);
+    }
     int rc = EVK_OK;
     if (cudaMemcpyAsync(ids_dev, ids_host, (size_t)M * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return EVK_ERR_CUDA;
@@ -586,6 +696,53 @@ int evk_q_update_host(evk_mem *mem, const int32_t *ids_host, int64_t M, int stag
         rc = EVK_ERR_CUDA;
     if (rc == EVK_OK)
         rc = evk_q_update(mem, ids_dev, M, stage, r_dev, alpha, inner, workspace_bytes - (size_t)(inner - ws), stream_v);
+    const cudaError_t sync = cudaStreamSynchronize(stream);
+    if (rc == EVK_OK && sync != cudaSuccess) rc = EVK_ERR_CUDA;
+    return rc;
+}
+
+size_t evk_mem_insert_host_workspace_bytes(const evk_mem *mem, int64_t n) {
+    if (!mem || n < 0) return 0;
+    return align256((size_t)n * mem->cfg.d * sizeof(float)) + align256((size_t)n * sizeof(float)) + 256;
+}
+
+int evk_mem_insert_host(evk_mem *mem, const void *emb_host, int emb_dtype, int64_t n, int stage,
+                        const float *q_init_host, void *workspace, size_t workspace_bytes, void *stream_v) {
+    // the host-side checks of evk_mem_insert, before anything is copied
+    if (!mem || n < 0 || (emb_dtype != EVK_DTYPE_F32 && emb_dtype != EVK_DTYPE_BF16)) return EVK_ERR_INVALID;
+    if (stage != EVK_STAGE_ALL && !stage_ok(mem, stage)) return EVK_ERR_INVALID;
+    if (n == 0) return EVK_OK;
+    if (!emb_host || !workspace || !aligned(workspace, 256)) return EVK_ERR_INVALID;
+    if (mem->size + n > mem->cfg.capacity) return EVK_ERR_CAPACITY;
+    if (workspace_bytes < evk_mem_insert_host_workspace_bytes(mem, n)) return EVK_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t e_bytes = (size_t)n * mem->cfg.d * (emb_dtype == EVK_DTYPE_F32 ? sizeof(float) : sizeof(__nv_bfloat16));
+    const size_t q_off = align256((size_t)n * mem->cfg.d * sizeof(float));
+    const size_t q_bytes = q_init_host ? (size_t)n * sizeof(float) : 0;
+    char *ws = static_cast<char *>(workspace);
+    const float *q_dev = q_init_host ? reinterpret_cast<const float *>(ws + q_off) : nullptr;
+    if (mem->stage_host && align256(e_bytes) + q_bytes <= mem->slot_bytes) {
+        // staged like evk_q_update_host: rows and start values leave through the page-locked slot
+        const int slot = acquire_slot(mem);
+        if (slot < 0) return EVK_ERR_CUDA;
+        char *h = mem->stage_host + (size_t)slot * mem->slot_bytes;
+        memcpy(h, emb_host, e_bytes);
+        if (q_bytes) memcpy(h + align256(e_bytes), q_init_host, q_bytes);
+        cudaError_t err = cudaMemcpyAsync(ws, h, e_bytes, cudaMemcpyHostToDevice, stream);
+        if (err == cudaSuccess && q_bytes)
+            err = cudaMemcpyAsync(ws + q_off, h + align256(e_bytes), q_bytes, cudaMemcpyHostToDevice, stream);
+        if (err != cudaSuccess || !release_slot_after(mem, slot, stream)) {
+            (void)cudaStreamSynchronize(stream);
+            return EVK_ERR_CUDA;
+        }
+        return evk_mem_insert(mem, ws, emb_dtype, n, stage, q_dev, nullptr, stream_v);
+    }
+    int rc = EVK_OK;
+    if (cudaMemcpyAsync(ws, emb_host, e_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return EVK_ERR_CUDA;
+    // a copy may be in flight from here on: every return synchronises first
+    if (q_bytes && cudaMemcpyAsync(ws + q_off, q_init_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        rc = EVK_ERR_CUDA;
+    if (rc == EVK_OK) rc = evk_mem_insert(mem, ws, emb_dtype, n, stage, q_dev, nullptr, stream_v);
     const cudaError_t sync = cudaStreamSynchronize(stream);
     if (rc == EVK_OK && sync != cudaSuccess) rc = EVK_ERR_CUDA;
     return rc;

@@ -43,7 +43,8 @@ EXPORTS = (
     "evk_mem_set_scoring", "evk_mem_set_score_norm", "evk_mem_inject_stall", "evk_mem_insert", "evk_retrieve_workspace_bytes", "evk_retrieve",
     "evk_q_update_workspace_bytes", "evk_q_update", "evk_q_update_static", "evk_q_update_decay", "evk_visits_read", "evk_visits_write", "evk_q_read", "evk_q_write", "evk_bank_read",
     "evk_retrieve_host_workspace_bytes", "evk_retrieve_host", "evk_q_update_host_workspace_bytes",
-    "evk_q_update_host", "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
+    "evk_q_update_host", "evk_mem_set_host_staging", "evk_mem_insert_host_workspace_bytes", "evk_mem_insert_host",
+    "evk_retrieve_plan", "evk_mem_profile_scoring", "evk_retrieve_explore_workspace_bytes",
     "evk_retrieve_explore", "evk_select_by_value", "evk_retrieve_local_workspace_bytes", "evk_retrieve_local",
     "evk_merge_shards", "evk_reward_draft",
     "evk_reward_refine", "evk_reward_norm_state_bytes", "evk_reward_norm_reset", "evk_reward_normalize", "evk_last_status",
@@ -103,6 +104,9 @@ def _load() -> ctypes.CDLL:
         "evk_retrieve_host": (cint, [vp, vp, cint, i32, cint, i32, i32, f32, vp, vp, vp, sz, vp]),
         "evk_q_update_host_workspace_bytes": (sz, [vp, i64]),
         "evk_q_update_host": (cint, [vp, vp, i64, cint, vp, f32, vp, sz, vp]),
+        "evk_mem_set_host_staging": (cint, [vp, vp, sz]),
+        "evk_mem_insert_host_workspace_bytes": (sz, [vp, i64]),
+        "evk_mem_insert_host": (cint, [vp, vp, cint, i64, cint, vp, vp, sz, vp]),
         "evk_retrieve_plan": (cint, [vp, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]),
         "evk_mem_profile_scoring": (cint, [vp, vp, vp]),
         "evk_retrieve_explore_workspace_bytes": (sz, [vp, i32, i32]),
@@ -185,6 +189,7 @@ class EvkMem:
         self.arena = arena
         self.d, self.capacity, self.n_stages = d, capacity, n_stages
         self._ws = {}
+        self.staging = None      # the page-locked tensor given to evk_mem_set_host_staging, kept alive here
 
     def workspace(self, kind: str, nbytes: int) -> torch.Tensor:
         """A cached scratch tensor of at least nbytes on the arena's device."""
@@ -398,6 +403,35 @@ def evk_retrieve_host(mem: EvkMem, queries_host: torch.Tensor, stage: int, k1: i
                                   _emb_dtype(queries_host), B, stage, k1, k2, float(w),
                                   _host(ids_out_host, torch.int32), _host(scores_out_host, torch.float32),
                                   _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_retrieve_host")
+
+
+def evk_mem_set_host_staging(mem: EvkMem, nbytes: int = 4 << 20) -> None:
+    """Give the bank a page-locked staging buffer of nbytes (0 withdraws it): evk_q_update_host and
+    evk_mem_insert_host then return without waiting for the device, and evk_retrieve_host receives
+    its result without a copy of its own."""
+    if nbytes <= 0:
+        _check(_lib.evk_mem_set_host_staging(mem.handle, None, 0), "evk_mem_set_host_staging")
+        mem.staging = None
+        return
+    # a torch allocation may start anywhere: over-allocate and hand over the 256-byte aligned part
+    buf = torch.empty(int(nbytes) + 256, dtype=torch.uint8).pin_memory()
+    skip = (-buf.data_ptr()) % 256
+    with torch.cuda.device(mem.arena.device):
+        _check(_lib.evk_mem_set_host_staging(mem.handle, buf.data_ptr() + skip, int(nbytes)), "evk_mem_set_host_staging")
+    mem.staging = buf
+
+
+def evk_mem_insert_host(mem: EvkMem, emb_host: torch.Tensor, stage: int = EVK_STAGE_ALL,
+                        q_init_host: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Host-buffer form of evk_mem_insert: the rows (and start values) are host tensors."""
+    if emb_host.dim() != 2 or emb_host.shape[1] != mem.d:
+        raise ValueError("emb_host must be [n][d]")
+    n = emb_host.shape[0]
+    nbytes = int(_lib.evk_mem_insert_host_workspace_bytes(mem.handle, n))
+    ws = mem.workspace("insert_host", nbytes)
+    _check(_lib.evk_mem_insert_host(mem.handle, _host(emb_host, None, "emb_host"), _emb_dtype(emb_host), n, stage,
+                                    _host(q_init_host, torch.float32, "q_init_host") if q_init_host is not None else None,
+                                    _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_mem_insert_host")
 
 
 def evk_q_update_host(mem: EvkMem, ids_host: torch.Tensor, stage: int, rewards_host: torch.Tensor,
