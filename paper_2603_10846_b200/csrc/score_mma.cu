@@ -84,15 +84,17 @@ constexpr int kChunk = 32;                           // accumulator columns per 
 // Self-starting histogram (scans of one query tile).  A similarity's bin is the top 13 bits of its
 // order-preserving bit pattern (sign, exponent, four mantissa bits: sixteen bins to the octave), so
 // every block bins alike without having seen any data; a query's 64 counters cover the window of
-// bins that the first block to finish its first tile anchors two octaves above that tile's largest
-// similarity (a first tile of 256 rows may miss the few entries that are much closer to the query than
+// bins that the first block to look at its first kBootCols rows anchors two octaves above those rows'
+// largest similarity (128 rows may miss the few entries that are much closer to the query than
 // the rest, as in a clustered bank).  Values above the window count in its top bin, values below it in bin 0, which never
 // serves as a threshold: a counter can only under-state how many entries reach its bin's edge.
 constexpr int kAbsShift = 19;
 constexpr int kAbsBins = 1 << (32 - kAbsShift);
 constexpr int kAbsHeadroom = 32;                     // bins between the anchoring maximum and the window's top
-constexpr int kBootBin = kHistBins - 1 - kAbsHeadroom - 16;   // first tile: entries from this window bin up (half the
-                                                     // anchoring maximum) are counted before any is filed
+constexpr int kBootCols = 128;                       // rows of a job's first tile that anchor the window and are counted
+constexpr int kBootBin = kHistBins - 1 - kAbsHeadroom - 16;   // ... from this window bin up (half the anchoring maximum)
+                                                     // before any entry is filed
+constexpr int kReadEvery = 4;                        // scans without a tracker: tiles between two looks at the counters
 constexpr int kSyncTiles = 4;                        // tiles of a job whose threshold the epilogue reads itself
 constexpr int kSyncAlways = 1 << 28;                 // ... or every tile: the tracker stays idle
 constexpr long long kTimeoutCycles = 4000000000LL;   // about two seconds
@@ -686,6 +688,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // self-starting histogram: window base (in absolute bins), whether this thread has one yet, and
             // the window bin from which this tile's entries were already counted ahead of filing
             int a_base = 0, skip_from = kHistBins;
+            int64_t counted_end = 0;   // first tile of a job: its rows below this were counted from bin skip_from up before filing
             bool anchored = false;
             if (q_valid) {
                 if (abs_mode) {
@@ -723,7 +726,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     }
                     if (key > tau_key && bin >= tau_bin) {
                         my_buf[cnt++] = key;
-                        if (my_hist && bin < skip_from && (anchored || !abs_mode)) atomicAdd(my_hist + bin, 1u);
+                        if (my_hist && (bin < skip_from || row >= counted_end) && (anchored || !abs_mode)) atomicAdd(my_hist + bin, 1u);
                     }
                 }
             };
@@ -804,36 +807,30 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
             };
             int sync_left = p.sync_tiles;
-            // self-starting histogram: the job's first tile is counted when it arrives but filed only when
-            // the second one is there (or the job ends); `held` says that its accumulator is still ours
-            bool held = false;
-            uint32_t held_acc = 0;
-            int64_t held_row0 = 0;
-            for (int t = split; ok; t += p.splits) {
-                const bool real = t < p.n_tiles;
-                if (!real && !held) break;
-                if (real) {
-                    if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
-                    tc_fence_after();
-                    if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
-                }
+            int n_done = 0;   // tiles of this job examined so far
+            for (int t = split; t < p.n_tiles && ok; t += p.splits, ++n_done) {
+                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                if (warp == 2 && lane == 0) *tile_seq = *tile_seq + 1;   // paces the tracker
                 uint32_t va[kChunk], vb[kChunk];
-                if (real && abs_mode && kMode == 0 && t == split) {
+                const int64_t row0 = (int64_t)t * kBlockN;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
+                skip_from = kHistBins;
+                counted_end = 0;
+                if (abs_mode && kMode == 0 && n_done == 0) {
                     // The job's first tile starts the histogram off (every lane of the warp walks through this,
-                    // the tensor-memory loads being warp-wide).  The window is anchored by whoever comes first,
-                    // and the tile's entries from window bin kBootBin up are counted.  Filing waits until the
-                    // next tile is in: by then every block has counted its first tile, and the counters give a
-                    // threshold that a few hundred of the 37,888 rows seen so far pass, where one block's own
-                    // 256 rows could justify none.  The tensor cores want this accumulator back only for the
-                    // third tile, whose rows arrive a whole tile later still.
-                    const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
-                    const int64_t row0 = (int64_t)t * kBlockN;
+                    // the tensor-memory loads being warp-wide).  Its first kBootCols rows anchor the window
+                    // (whoever comes first) and are counted from window bin kBootBin up; then the tile is filed
+                    // like any other.  All blocks start together, so by the time this one reads the counters
+                    // most of the others have counted their first rows too, and the counters give a threshold
+                    // that a few hundred of the 18,944 rows counted pass, where one block's own rows could
+                    // justify none (a threshold from fewer counts is lower, never wrong).
                     int enc = my_hist ? __ldcg(p.anchor + q) : 1;
                     if (__any_sync(0xffffffffu, enc == 0)) {
-                        // nobody has anchored this query's window yet: this tile's largest similarity does
+                        // nobody has anchored this query's window yet: these rows' largest similarity does
                         float mx = -INFINITY;
 #pragma unroll 1
-                        for (int c0 = 0; c0 < kBlockN; c0 += kChunk) {
+                        for (int c0 = 0; c0 < kBootCols; c0 += kChunk) {
                             tmem_ld_issue(t_addr + c0, va);
                             tmem_ld_wait(va);
 #pragma unroll
@@ -853,15 +850,11 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         a_base = enc - 1;
                         anchored = true;
                     }
-                    tmem_ld_issue(t_addr, va);
-                    tmem_ld_wait(va);
                     const float cnt_edge = anchored ? from_ordered_bits((uint32_t)(a_base + kBootBin) << kAbsShift) : INFINITY;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kBlockN; c0 += kChunk) {
-                        if (c0 > 0) {
-                            tmem_ld_issue(t_addr + c0, va);
-                            tmem_ld_wait(va);
-                        }
+                    for (int c0 = 0; c0 < kBootCols; c0 += kChunk) {
+                        tmem_ld_issue(t_addr + c0, va);
+                        tmem_ld_wait(va);
                         uint32_t bits[kChunk];
 #pragma unroll
                         for (int j = 0; j < kChunk; ++j) bits[j] = __uint_as_float(va[j]) >= cnt_edge ? (1u << j) : 0u;
@@ -881,61 +874,51 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                             }
                         }
                     }
-                    held = true;
-                    held_acc = acc;
-                    held_row0 = row0;
-                    if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-                    continue;
+                    // the counted rows' entries from kBootBin up are in the counters already
+                    if (anchored) {
+                        skip_from = kBootBin;
+                        counted_end = row0 + kBootCols;
+                    }
                 }
-                // the tile held back first (if any), then the one that has just arrived (if any)
+                // At the start of a job a threshold moves with every tile and the tracker's word comes
+                // a tile late: there the thread reads its counters itself, later it takes the word.  A scan
+                // without a tracker keeps reading them, every tile at first and every kReadEvery-th after that:
+                // all blocks read the same one or two L2 lines per query, the very lines the survivors' atomic
+                // updates go to, and reading them for every tile slowed the whole scan (2 GiB, 128 queries:
+                // 0.38-0.39 against 0.357 ms; 64 queries: 5-10 us; the lists grow by 2 %).
+                if (sync_left > 0 && (n_done < kReadEvery || n_done % kReadEvery == 0)) {
+                    --sync_left;
+                    // (sampled thresholds: nothing to read before the block's very first tile, every block
+                    // starts at once and the counters are still empty)
+                    if (my_hist && (abs_mode ? anchored : !(job == worker && n_done == 0)))
+                        raise_bin(hist_best_bin(my_hist, p.k1));
+                } else {
+                    refresh();
+                }
+                // two register buffers: the next chunk's load is in flight while one is examined
+                tmem_ld_issue(t_addr, va);
+                tmem_ld_wait(va);
 #pragma unroll 1
-                for (int rep = held ? 0 : 1; rep < (real ? 2 : 1); ++rep) {
-                    const bool old = rep == 0;
-                    const uint32_t use_acc = old ? held_acc : acc;
-                    const int64_t row0 = old ? held_row0 : (int64_t)t * kBlockN;
-                    // entries of the held tile from kBootBin up are in the counters already
-                    skip_from = (old && anchored) ? kBootBin : kHistBins;
-                    // At the start of a job a threshold moves with every tile and the tracker's word comes
-                    // a tile late: there the thread reads its counters itself, later it takes the word.
-                    if (sync_left > 0) {
-                        if (!old) --sync_left;
-                        // (sampled thresholds: nothing to read before the block's very first tile, every block
-                        // starts at once and the counters are still empty)
-                        if (my_hist && (abs_mode ? anchored : !(job == worker && t == split)))
-                            raise_bin(hist_best_bin(my_hist, p.k1));
-                    } else {
-                        refresh();
-                    }
-                    const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + use_acc * kBlockN;
-                    // two register buffers: the next chunk's load is in flight while one is examined
-                    tmem_ld_issue(t_addr, va);
-                    tmem_ld_wait(va);
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kBlockN - 2 * kChunk; c0 += 2 * kChunk) {
-                        tmem_ld_issue(t_addr + c0 + kChunk, vb);
-                        process(va, row0, c0);
-                        tmem_ld_wait(vb);
-                        tmem_ld_issue(t_addr + c0 + 2 * kChunk, va);
-                        refresh();
-                        process(vb, row0, c0 + kChunk);
-                        tmem_ld_wait(va);
-                    }
-                    tmem_ld_issue(t_addr + kBlockN - kChunk, vb);
-                    process(va, row0, kBlockN - 2 * kChunk);
+                for (int c0 = 0; c0 < kBlockN - 2 * kChunk; c0 += 2 * kChunk) {
+                    tmem_ld_issue(t_addr + c0 + kChunk, vb);
+                    process(va, row0, c0);
                     tmem_ld_wait(vb);
-                    // every column of this accumulator is in registers: hand it back before the last look
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * use_acc, 0)); else mbar_arrive(tempty0 + 8 * use_acc);
-                    }
-                    if (!old) {
-                        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-                    }
-                    process(vb, row0, kBlockN - kChunk);
+                    tmem_ld_issue(t_addr + c0 + 2 * kChunk, va);
+                    refresh();
+                    process(vb, row0, c0 + kChunk);
+                    tmem_ld_wait(va);
                 }
-                held = false;
-                if (!real) break;
+                tmem_ld_issue(t_addr + kBlockN - kChunk, vb);
+                process(va, row0, kBlockN - 2 * kChunk);
+                tmem_ld_wait(vb);
+                // every column of this accumulator is in registers: hand it back before the last look
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (kPair) mbar_arrive_cluster(mapa_u32(tempty0 + 8 * acc, 0)); else mbar_arrive(tempty0 + 8 * acc);
+                }
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                process(vb, row0, kBlockN - kChunk);
             }
             if (kMode == 0 && ok && qt < p.n_qt && row >= 0) p.cand_cnt[(size_t)list_job * kBlockM + row] = cnt;
             if (kMode == 0 && p.dev) {
