@@ -1453,9 +1453,11 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         p.a_resident = 0;
         p.a_rows = kBlockM;
         // four stages here too: the same speed as six on short scans, 5 % faster on the long
-        // power-capped one (19.7 against 20.7 ms for 4,096 queries over 6 GiB)
-        p.n_stages = kResidentStages;
-        smem_bytes = kSmemFixed + (size_t)kResidentStages * (kABytes + kBBytes / 2);
+        // power-capped one (19.7 against 20.7 ms for 4,096 queries over 6 GiB).  One pair of query tiles
+        // is bound by HBM instead, and four stages of 16 KB of bank rows keep too few bytes in flight:
+        // six there (129-256 queries over 2 GiB: 0.433-0.493 -> 0.410-0.472 ms)
+        p.n_stages = pl.n_qt <= 2 ? kMaxStages : kResidentStages;
+        smem_bytes = kSmemFixed + (size_t)p.n_stages * (kABytes + kBBytes / 2);
     }
     p.size = size;
     p.mode = 0;
