@@ -149,9 +149,15 @@ def _check(status: int, where: str) -> None:
         raise EvkError(status, where)
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    s = stream if stream is not None else torch.cuda.current_stream()
-    return int(s.cuda_stream)
+    if stream is not None:
+        return int(stream.cuda_stream)
+    if _raw_stream is not None:      # the current stream's handle without building a Stream object
+        return int(_raw_stream(torch.cuda.current_device()))
+    return int(torch.cuda.current_stream().cuda_stream)
 
 
 def _dev(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
@@ -189,7 +195,16 @@ class EvkMem:
         self.arena = arena
         self.d, self.capacity, self.n_stages = d, capacity, n_stages
         self._ws = {}
+        self._ws_bytes = {}
         self.staging = None      # the page-locked tensor given to evk_mem_set_host_staging, kept alive here
+
+    def workspace_for(self, kind: str, key, size_fn) -> torch.Tensor:
+        """The scratch tensor of one call shape; the library is asked for its size once per shape
+        (sizes depend on the shape, the bank's capacity and the scoring mode only)."""
+        nbytes = self._ws_bytes.get((kind, key))
+        if nbytes is None:
+            nbytes = self._ws_bytes[(kind, key)] = int(size_fn())
+        return self.workspace(kind, nbytes)
 
     def workspace(self, kind: str, nbytes: int) -> torch.Tensor:
         """A cached scratch tensor of at least nbytes on the arena's device."""
@@ -241,6 +256,7 @@ def evk_launch_count(mem: EvkMem) -> int:
 
 def evk_mem_set_scoring(mem: EvkMem, mode: int) -> None:
     _check(_lib.evk_mem_set_scoring(mem.handle, mode), "evk_mem_set_scoring")
+    mem._ws_bytes.clear()
 
 
 def evk_mem_set_score_norm(mem: EvkMem, mode: int) -> None:
@@ -279,7 +295,7 @@ def evk_retrieve(mem: EvkMem, queries: torch.Tensor, stage: int, k1: int, k2: in
     pool_ids = torch.empty((B, k1), dtype=torch.int32, device=dev) if return_pool else None
     pool_sims = torch.empty((B, k1), dtype=torch.float32, device=dev) if return_pool else None
     if workspace is None:
-        workspace = mem.workspace("retrieve", evk_retrieve_workspace_bytes(mem, B, k1))
+        workspace = mem.workspace_for("retrieve", (B, k1), lambda: _lib.evk_retrieve_workspace_bytes(mem.handle, B, k1))
     _check(_lib.evk_retrieve(mem.handle, _dev(queries, None, "queries"), _emb_dtype(queries), B, stage,
                              k1, k2, float(w), _dev(ids, torch.int32), _dev(scores, torch.float32),
                              _dev(pool_ids), _dev(pool_sims),
@@ -300,7 +316,7 @@ def evk_q_update(mem: EvkMem, ids: torch.Tensor, stage: int, rewards: torch.Tens
     if rewards.numel() != M:
         raise ValueError("ids and rewards must have the same length")
     if workspace is None:
-        workspace = mem.workspace("q_update", evk_q_update_workspace_bytes(mem, M))
+        workspace = mem.workspace_for("q_update", M, lambda: _lib.evk_q_update_workspace_bytes(mem.handle, M))
     _check(_lib.evk_q_update(mem.handle, _dev(ids, torch.int32, "ids"), M, stage,
                              _dev(rewards, torch.float32, "rewards"), float(alpha),
                              _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)),
@@ -397,8 +413,8 @@ def evk_retrieve_host(mem: EvkMem, queries_host: torch.Tensor, stage: int, k1: i
                       ids_out_host: torch.Tensor, scores_out_host: torch.Tensor, stream=None) -> None:
     """Host-buffer form: copies queries in and results out inside the call, then synchronises."""
     B = queries_host.shape[0]
-    nbytes = int(_lib.evk_retrieve_host_workspace_bytes(mem.handle, B, k1, k2))
-    ws = mem.workspace("retrieve_host", nbytes)
+    ws = mem.workspace_for("retrieve_host", (B, k1, k2),
+                           lambda: _lib.evk_retrieve_host_workspace_bytes(mem.handle, B, k1, k2))
     _check(_lib.evk_retrieve_host(mem.handle, _host(queries_host, None, "queries_host"),
                                   _emb_dtype(queries_host), B, stage, k1, k2, float(w),
                                   _host(ids_out_host, torch.int32), _host(scores_out_host, torch.float32),
@@ -427,8 +443,7 @@ def evk_mem_insert_host(mem: EvkMem, emb_host: torch.Tensor, stage: int = EVK_ST
     if emb_host.dim() != 2 or emb_host.shape[1] != mem.d:
         raise ValueError("emb_host must be [n][d]")
     n = emb_host.shape[0]
-    nbytes = int(_lib.evk_mem_insert_host_workspace_bytes(mem.handle, n))
-    ws = mem.workspace("insert_host", nbytes)
+    ws = mem.workspace_for("insert_host", n, lambda: _lib.evk_mem_insert_host_workspace_bytes(mem.handle, n))
     _check(_lib.evk_mem_insert_host(mem.handle, _host(emb_host, None, "emb_host"), _emb_dtype(emb_host), n, stage,
                                     _host(q_init_host, torch.float32, "q_init_host") if q_init_host is not None else None,
                                     _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_mem_insert_host")
@@ -437,8 +452,7 @@ def evk_mem_insert_host(mem: EvkMem, emb_host: torch.Tensor, stage: int = EVK_ST
 def evk_q_update_host(mem: EvkMem, ids_host: torch.Tensor, stage: int, rewards_host: torch.Tensor,
                       alpha: float, stream=None) -> None:
     M = ids_host.numel()
-    nbytes = int(_lib.evk_q_update_host_workspace_bytes(mem.handle, M))
-    ws = mem.workspace("q_update_host", nbytes)
+    ws = mem.workspace_for("q_update_host", M, lambda: _lib.evk_q_update_host_workspace_bytes(mem.handle, M))
     _check(_lib.evk_q_update_host(mem.handle, _host(ids_host, torch.int32), M, stage,
                                   _host(rewards_host, torch.float32), float(alpha),
                                   _dev(ws), ws.numel(), _stream_ptr(stream)), "evk_q_update_host")
