@@ -240,6 +240,14 @@ constexpr uint32_t kInstrDescSub = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32
 constexpr uint32_t kInstrDescSubM64 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSubRows >> 3) << 17) |
                                       ((uint32_t)(64 >> 4) << 24);
 
+// Swapped roles for up to kSwapN queries: the bank rows are the M side (128 of them per instruction, one
+// per accumulator lane), the queries the N side, padded to kSwapN instead of to 64: a quarter of the
+// tensor work per bank row.  The scan is bound by HBM either way; under the power cap the tensor cores'
+// share of the board's power is what sets the clock, and padding rows cost as much as real ones.
+constexpr int kSwapN = 16;
+constexpr uint32_t kInstrDescSwap = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSwapN >> 3) << 17) |
+                                    ((uint32_t)(kSubRows >> 4) << 24);
+
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
                                           uint32_t idesc) {
     asm volatile(
@@ -340,6 +348,23 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.wait::ld.sync.aligned;"
         : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+        :
+        : "memory");
+}
+
+// Sixteen columns (the swapped layout: one column per query).
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
         :
         : "memory");
 }
@@ -453,7 +478,220 @@ __device__ __noinline__ uint64_t warp_select_topk(uint64_t *buf, int n, int k) {
 // (scans of one query tile) instead of sampled ones.  Three shapes are built: <false, 0, true>,
 // <true, 0, false> and <false, 1, false>; each carries only its own code (the epilogue's speed
 // depends on how much code it has to run through).
-template <bool kPair, int kMode, bool kAbs>
+// ---- epilogue of the swapped layout (up to kSwapN queries) ---------------------------------------
+// A thread owns one bank row of each 128-row group (its accumulator lane) and holds that row's
+// similarity to every query in registers; what is per query lives in shared memory, shared by the four
+// epilogue warps: list length, thresholds, histogram window.  Query j is looked after by warp j % 4
+// (threshold reads, cut-backs).  The warps meet at a named barrier between the phases of a tile; every
+// branch around such a barrier is taken by all four alike (a failed wait is published through a flag
+// that all read behind the next barrier, see `fail`).
+struct SwapState {
+    int cnt[kSwapN];              // candidates in the job's list of query j
+    int tau_bin[kSwapN];          // bin threshold from the shared histogram
+    float tau_sim[kSwapN];        // cheap first test: no larger than either exact threshold
+    float floor_sim[kSwapN];      // similarity of tau_key
+    uint64_t tau_key[kSwapN];     // exact key threshold (rises when the list is cut back)
+    int a_base[kSwapN];           // lowest absolute bin of the window, -1 until anchored
+    unsigned mx[kSwapN];          // first rows' largest similarity as ordered bits (start-up)
+    int fail[2];                  // a wait ran out in a round of this parity
+};
+static_assert(sizeof(SwapState) <= 1536, "lives in the tracker's mailboxes, which this layout leaves unused");
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Highest bin of the histogram with k1 counted entries at or above it (0: none yet); the whole warp
+// reads the 64 counters, two per lane.
+__device__ __forceinline__ int warp_best_bin(const unsigned *hist, int k1, int lane) {
+    const uint2 c = __ldcg(reinterpret_cast<const uint2 *>(hist) + lane);
+    int own = (int)(c.x + c.y), incl = own;   // incl: this lane's counters and all higher ones
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += v;
+    }
+    const int above = incl - own;
+    const bool here = above < k1 && k1 <= incl;
+    const unsigned who = __ballot_sync(0xffffffffu, here);
+    if (!who) return 0;
+    const int src = __ffs(who) - 1;
+    const int bin = (above + (int)c.y >= k1) ? 2 * lane + 1 : 2 * lane;
+    return __shfl_sync(0xffffffffu, bin, src);
+}
+
+// Returns false when a wait ran out (the block then backs out like the other layouts).
+__device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st, uint32_t tmem_base, uint32_t tfull0,
+                                              uint32_t tempty0, volatile int *abort_flag, long long wait_limit,
+                                              int warp, int lane, int worker, int n_jobs, int n_workers) {
+    const int quarter = warp & 3;            // this warp's tensor-memory lanes: 32 * quarter ...
+    const int tid128 = quarter * 32 + lane;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    uint32_t acc = 0, acc_phase = 0;
+    int round = 0;
+    bool ok = true;
+    if (tid128 == 0) st->fail[0] = st->fail[1] = 0;
+    for (int job = worker; job < n_jobs && ok; job += n_workers) {
+        const int split = job % p.splits;    // one query tile: the job is the bank split
+        if (tid128 < kSwapN) {
+            st->cnt[tid128] = 0;
+            st->tau_bin[tid128] = 0;
+            st->tau_sim[tid128] = -INFINITY;
+            st->floor_sim[tid128] = -INFINITY;
+            st->tau_key[tid128] = 0;
+            st->a_base[tid128] = -1;
+            st->mx[tid128] = 0;
+        }
+        epi_bar();
+        int n_done = 0;
+        for (int t = split; t < p.n_tiles; t += p.splits, ++n_done) {
+            if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) st->fail[round & 1] = 1;
+            epi_bar();
+            if (st->fail[round & 1]) { ok = false; break; }
+            ++round;
+            tc_fence_after();
+            uint32_t v0[kSwapN], v1[kSwapN];   // this thread's row of group 0 and of group 1 against every query
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
+            tmem_ld16_issue(t_addr, v0);
+            tmem_ld16_issue(t_addr + kSwapN, v1);
+            tmem_ld16_wait(v0);
+            tmem_ld16_wait(v1);
+            // the whole accumulator is in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            const int64_t row_a = (int64_t)t * kBlockN + tid128, row_b = row_a + kSubRows;
+            const bool live_a = row_a < p.size && entry_live(p.live_bits, row_a);
+            const bool live_b = row_b < p.size && entry_live(p.live_bits, row_b);
+            int skip_from = kHistBins;
+            int64_t counted_end = 0;
+            if (n_done == 0) {
+                // The job's first 128 rows start the histogram off: their largest similarity anchors each
+                // query's window (whoever comes first), and those of them from window bin kBootBin up are
+                // counted before anything is filed (see the other layout's epilogue).
+#pragma unroll
+                for (int j = 0; j < kSwapN; ++j) {
+                    if (j < p.B) {
+                        const float x = __uint_as_float(v0[j]);
+                        const unsigned ob = (row_a < p.size && fabsf(x) <= 3.0e38f) ? ordered_bits(x + 0.0f) : 0u;
+                        const unsigned wm = __reduce_max_sync(0xffffffffu, ob);
+                        if (lane == 0 && wm) atomicMax(&st->mx[j], wm);
+                    }
+                }
+                epi_bar();
+                for (int j = quarter; j < p.B; j += 4) {
+                    if (lane == 0) {
+                        int enc = __ldcg(p.anchor + j);
+                        if (enc == 0 && st->mx[j] != 0) {
+                            int prop = (int)(st->mx[j] >> kAbsShift) + kAbsHeadroom - (kHistBins - 1);
+                            prop = prop < 0 ? 0 : (prop > kAbsBins - kHistBins ? kAbsBins - kHistBins : prop);
+                            const int got = atomicCAS(p.anchor + j, 0, prop + 1);
+                            enc = got ? got : prop + 1;
+                        }
+                        if (enc != 0) st->a_base[j] = enc - 1;
+                    }
+                }
+                epi_bar();
+#pragma unroll
+                for (int j = 0; j < kSwapN; ++j) {
+                    if (j < p.B) {
+                        const int ab = st->a_base[j];
+                        const float x = __uint_as_float(v0[j]);
+                        if (ab >= 0 && live_a && x >= from_ordered_bits((uint32_t)(ab + kBootBin) << kAbsShift)) {
+                            int bin = (int)(ordered_bits(x + 0.0f) >> kAbsShift) - ab;
+                            bin = bin > kHistBins - 1 ? kHistBins - 1 : bin;
+                            atomicAdd(p.hist + (size_t)j * kHistBins + bin, 1u);
+                        }
+                    }
+                }
+                skip_from = kBootBin;
+                counted_end = (int64_t)t * kBlockN + kBootCols;
+                epi_bar();
+            }
+            // the thresholds: read before each of the first tiles, then before every kReadEvery-th
+            if (n_done < kReadEvery || n_done % kReadEvery == 0) {
+                for (int j = quarter; j < p.B; j += 4) {
+                    const int ab = st->a_base[j];
+                    if (ab >= 0) {
+                        const int best = warp_best_bin(p.hist + (size_t)j * kHistBins, p.k1, lane);
+                        if (lane == 0 && best > st->tau_bin[j]) {
+                            st->tau_bin[j] = best;
+                            st->tau_sim[j] = fmaxf(st->floor_sim[j], from_ordered_bits((uint32_t)(ab + best) << kAbsShift));
+                        }
+                    }
+                }
+                epi_bar();
+            }
+            // file what passes: one ballot per query and row group, the list's slots claimed per warp
+            auto file_one = [&](uint32_t bits, int64_t row, bool live, int j) {
+                const float sv = __uint_as_float(bits);
+                bool pass = live && sv >= st->tau_sim[j];
+                uint64_t key = 0;
+                int bin = 0;
+                const int ab = st->a_base[j];
+                if (pass) {
+                    key = make_key(sv, (int32_t)row);
+                    if (ab >= 0) {
+                        bin = (int)(ordered_bits(sv + 0.0f) >> kAbsShift) - ab;
+                        bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
+                    }
+                    pass = key > st->tau_key[j] && bin >= st->tau_bin[j];
+                }
+                const unsigned m = __ballot_sync(0xffffffffu, pass);
+                if (m) {
+                    const int first = __ffs(m) - 1;
+                    int base = 0;
+                    if (lane == first) base = atomicAdd(&st->cnt[j], __popc(m));
+                    base = __shfl_sync(0xffffffffu, base, first);
+                    if (pass) {
+                        p.cand[((size_t)split * kBlockM + j) * kMmaCandCap + base + __popc(m & lt_mask)] = key;
+                        // (entries of the counted first rows from kBootBin up are in the counters already)
+                        if (ab >= 0 && (bin < skip_from || row >= counted_end))
+                            atomicAdd(p.hist + (size_t)j * kHistBins + bin, 1u);
+                    }
+                }
+            };
+#pragma unroll
+            for (int j = 0; j < kSwapN; ++j) {
+                if (j < p.B) {
+                    file_one(v0[j], row_a, live_a, j);
+                    file_one(v1[j], row_b, live_b, j);
+                }
+            }
+            // a list that the next tile could overflow (256 rows may all pass) is cut back to its best k1
+            epi_bar();
+            for (int j = quarter; j < p.B; j += 4) {
+                const int n = st->cnt[j];
+                if (n > kMmaCandCap - kBlockN) {
+                    const uint64_t kth = warp_select_topk(p.cand + ((size_t)split * kBlockM + j) * kMmaCandCap, n, p.k1);
+                    if (lane == 0) {
+                        if (p.dev) atomicAdd(p.dev + kDevCutbacks, 1u);
+                        st->cnt[j] = p.k1;
+                        st->tau_key[j] = kth;
+                        st->floor_sim[j] = key_sim(kth);
+                        st->tau_sim[j] = fmaxf(st->tau_sim[j], st->floor_sim[j]);
+                    }
+                }
+            }
+            epi_bar();
+        }
+        epi_bar();
+        if (tid128 < p.B) p.cand_cnt[(size_t)split * kBlockM + tid128] = ok ? st->cnt[tid128] : 0;
+        if (p.dev && ok && tid128 == 0) {
+            unsigned long long left = 0;
+            for (int j = 0; j < p.B; ++j) left += (unsigned long long)st->cnt[j];
+            if (left) atomicAdd(reinterpret_cast<unsigned long long *>(p.dev + kDevFiledLo), left);
+        }
+        epi_bar();
+    }
+    if (!ok) {
+        // backing out: whatever this block was to deliver counts as empty, so the merge reads nothing stale
+        for (int job = worker; job < n_jobs; job += n_workers)
+            if (tid128 < p.B) p.cand_cnt[(size_t)(job % p.splits) * kBlockM + tid128] = 0;
+    }
+    return ok;
+}
+
+template <bool kPair, int kMode, bool kAbs, bool kSwap = false>
 __global__ void __launch_bounds__(kThreads, 1)
 score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
                  const MmaParams p) {
@@ -627,9 +865,14 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                     const uint64_t a_desc = smem_desc(tiles + kc * a_slice);
                                     const uint64_t b_desc = smem_desc(s_addr + sl * (kSubRows * 128));
 #pragma unroll
-                                    for (int k = 0; k < kBlockK / kUmmaK; ++k)
-                                        umma_bf16(d_tmem + g * kSubRows, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
-                                                  (kc > 0 || k > 0) ? 1u : 0u, idesc);
+                                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                                        if (kSwap)   // bank rows on the lanes, row group g in columns [16 g, 16 g + 16)
+                                            umma_bf16(d_tmem + g * kSwapN, b_desc + (uint64_t)(2 * k), a_desc + (uint64_t)(2 * k),
+                                                      (kc > 0 || k > 0) ? 1u : 0u, kInstrDescSwap);
+                                        else
+                                            umma_bf16(d_tmem + g * kSubRows, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                                      (kc > 0 || k > 0) ? 1u : 0u, idesc);
+                                    }
                                 }
                             }
                             umma_commit(empty0 + 8 * stage);
@@ -665,6 +908,12 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // The thresholds, the histogram and the candidate lists belong to the kernels before this
         // one; loads and MMAs of the first tiles run ahead while the epilogue waits for them.
         pdl_wait();
+        if constexpr (kSwap) {
+            SwapState *st = reinterpret_cast<SwapState *>(reinterpret_cast<unsigned char *>(bars) + 256);
+            swap_epilogue(p, st, tmem_base, tfull0, tempty0, abort_flag, wait_limit, warp, lane, worker, n_jobs, n_workers);
+            __syncwarp();
+            if (lane == 0) atomicAdd(const_cast<int *>(epi_done), 1);
+        } else {
         const int quarter = warp & 3;              // warps 2,3,4,5 -> lane quarters 2,3,0,1
         const int m = quarter * 32 + lane;
         // the tile's row on this lane: m itself, or with M = 64 sixteen rows per quarter (none on lanes 16-31)
@@ -938,6 +1187,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         __syncwarp();
         if (lane == 0) atomicAdd(const_cast<int *>(epi_done), 1);
+        }
     } else {
         // ===== threshold tracker: lane l looks after epilogue threads l, l+32, l+64, l+96 =====
         // The counters are read on a thinning schedule: after every tile at the start of a job,
@@ -1217,7 +1467,8 @@ struct SmemPlan {
 
 SmemPlan smem_plan(int B, int d) {
     SmemPlan sp;
-    const int rows = B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM;
+    // up to kSwapN queries of whole slices go to the swapped layout, whose query tile has kSwapN rows
+    const int rows = (B <= kSwapN && d % kBlockK == 0) ? kSwapN : (B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM);
     const size_t a_bytes = (size_t)rows * ((d + kBlockK - 1) / kBlockK * kBlockK) * 2;
     const size_t budget = kSmemMax - kSmemFixed;
     if (B <= kBlockM && a_bytes + 3 * (size_t)kBBytes <= budget) {
@@ -1240,9 +1491,10 @@ SmemPlan smem_plan(int B, int d) {
 // overlap = true: programmatic dependent launch behind the kernel enqueued just before.
 // pair = true: clusters of two blocks (grid must be even), the cta_group::2 variant.
 cudaError_t launch_kernel(const CUtensorMap &mq, const CUtensorMap &mb, const MmaParams &p, int grid,
-                          size_t smem_bytes, bool overlap, bool pair, cudaStream_t stream) {
+                          size_t smem_bytes, bool overlap, bool pair, cudaStream_t stream, bool swap = false) {
     auto kern = pair ? score_mma_kernel<true, 0, false>
-                     : (p.mode == 1 ? score_mma_kernel<false, 1, false> : score_mma_kernel<false, 0, true>);
+                     : (p.mode == 1 ? score_mma_kernel<false, 1, false>
+                                    : (swap ? score_mma_kernel<false, 0, true, true> : score_mma_kernel<false, 0, true>));
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -1400,7 +1652,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     // Up to 64 resident queries: M = 64 instructions.  The scan is bound by HBM either way, but the
     // tensor cores then do half the work on padding rows, and under the power cap that is worth
     // 250 MHz of SM clock and 4-5 % of a step (0.398 against 0.420 ms at 64 queries over 2 GiB).
-    p.m64 = (sp.a_resident && sp.a_rows <= 64) ? 1 : 0;
+    p.m64 = (sp.a_resident && sp.a_rows <= 64) ? 1 : 0;   // (the swapped layout has its own instruction shape)
     p.a_rows = sp.a_rows;
     p.n_stages = sp.n_stages;
     // resident queries and a width of whole slices: bank stages of 64 rows x 4 slices
@@ -1477,7 +1729,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         // attribute was seen, on B200 with driver 580, to run past its griddepcontrol.wait while its
         // predecessor was still running, so the paired scan is launched in plain stream order.)
         err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, p.abs_hist && !pl.pair && !ev_start,
-                            pl.pair != 0, stream);
+                            pl.pair != 0, stream, !pl.pair && p.b3d && B <= kSwapN);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);

@@ -604,6 +604,23 @@ def test_tensor_path_candidate_lists_overflow_and_are_cut_back(evk):
     parity.check_retrieve(host_bits(bank2), host_bits(queries), q_tab[0], k1, 10, 0.5, out2, sample=[0, 1, 1999])
 
 
+def test_few_queries_lists_overflow_and_are_cut_back(evk):
+    # up to 16 queries take the layout with the bank rows on the accumulator lanes; a bank sorted against
+    # the scan for query 0 makes every row of every tile pass, so that its lists fill and are cut back
+    n, d, b, k1 = 250000, 64, 3, 100
+    bank = synth.gaussian_unit(n, d, 97, DEV)
+    queries = synth.gaussian_unit(b, d, 98, DEV)
+    order = torch.argsort((bank.float() @ queries[:1].float().T).squeeze(1))
+    bank = bank[order].contiguous()
+    q_tab = np.random.default_rng(8).random((2, n)).astype(np.float32)
+    mem = make_mem(evk, bank, q_tab, scoring=evk.EVK_SCORING_TENSOR)
+    before = evk.evk_mem_stats(mem)["list_cutbacks"]
+    out = run_retrieve(evk, mem, queries, 0, k1, 10, 0.5)
+    assert evk.evk_mem_stats(mem)["list_cutbacks"] > before
+    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, 10, 0.5, out)
+    assert ep == 1.0 and ef == 1.0
+
+
 def test_more_query_tiles_than_sms(evk):
     # 149 query tiles: each gets a single bank split and blocks take several jobs in turn
     n, d, b, k1 = 3000, 64, 149 * 128 - 5, 20
@@ -617,10 +634,11 @@ def test_more_query_tiles_than_sms(evk):
     assert ep >= 0.9 and ef >= 0.9
 
 
-@pytest.mark.parametrize("b", [20, 200, 330])
+@pytest.mark.parametrize("b", [5, 20, 200, 330])
 def test_bounded_wait_runs_out_and_the_handle_survives(evk, b):
     # failure detection without a fault: the producer of one scan issues no loads, the consumer's
-    # wait expires, every block backs out, and the status word says so.  20 queries: single blocks;
+    # wait expires, every block backs out, and the status word says so.  5 queries: single blocks with
+    # the bank rows on the accumulator lanes (four epilogue warps leave together); 20: single blocks;
     # 200: one pair of blocks per tile; 330: a second pair whose other block has a tile of padding
     n, d = 40000, 256
     bank = synth.gaussian_unit(n, d, 101, DEV)
