@@ -240,13 +240,19 @@ constexpr uint32_t kInstrDescSub = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32
 constexpr uint32_t kInstrDescSubM64 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSubRows >> 3) << 17) |
                                       ((uint32_t)(64 >> 4) << 24);
 
-// Swapped roles for up to kSwapN queries: the bank rows are the M side (128 of them per instruction, one
-// per accumulator lane), the queries the N side, padded to kSwapN instead of to 64: a quarter of the
-// tensor work per bank row.  The scan is bound by HBM either way; under the power cap the tensor cores'
+// Swapped roles for up to kSwapMax queries: the bank rows are the M side (128 of them per instruction, one
+// per accumulator lane), the queries the N side, padded to a multiple of kSwapN instead of to 64: as
+// little as a quarter of the tensor work per bank row.  The scan is bound by HBM either way; under the power cap the tensor cores'
 // share of the board's power is what sets the clock, and padding rows cost as much as real ones.
-constexpr int kSwapN = 16;
-constexpr uint32_t kInstrDescSwap = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kSwapN >> 3) << 17) |
-                                    ((uint32_t)(kSubRows >> 4) << 24);
+constexpr int kSwapN = 16;                           // queries per chunk of the epilogue, granularity of N
+#ifndef EVK_SWAP_MAX
+#define EVK_SWAP_MAX 32
+#endif
+constexpr int kSwapMax = EVK_SWAP_MAX;               // most queries this layout takes
+__host__ __device__ constexpr int swap_n(int B) { return ((B + kSwapN - 1) / kSwapN) * kSwapN; }
+__device__ __forceinline__ uint32_t instr_desc_swap(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kSubRows >> 4) << 24);
+}
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
                                           uint32_t idesc) {
@@ -486,14 +492,12 @@ __device__ __noinline__ uint64_t warp_select_topk(uint64_t *buf, int n, int k) {
 // branch around such a barrier is taken by all four alike (a failed wait is published through a flag
 // that all read behind the next barrier, see `fail`).
 struct SwapState {
-    int cnt[kSwapN];              // candidates in the job's list of query j
-    int tau_bin[kSwapN];          // bin threshold from the shared histogram
-    float tau_sim[kSwapN];        // cheap first test: no larger than either exact threshold
-    float floor_sim[kSwapN];      // similarity of tau_key
-    uint64_t tau_key[kSwapN];     // exact key threshold (rises when the list is cut back)
-    int a_base[kSwapN];           // lowest absolute bin of the window, -1 until anchored
-    unsigned mx[kSwapN];          // first rows' largest similarity as ordered bits (start-up)
-    int fail[2];                  // a wait ran out in a round of this parity
+    int cnt[kSwapMax];            // candidates in the job's list of query j (at a job's start: the first rows'
+                                  // largest similarity as ordered bits, until the window is anchored)
+    int tau_bin[kSwapMax];        // bin threshold from the shared histogram
+    float tau_sim[kSwapMax];      // cheap first test: no larger than either exact threshold
+    uint64_t tau_key[kSwapMax];   // exact key threshold (rises when the list is cut back)
+    int a_base[kSwapMax];         // lowest absolute bin of the window, -1 until anchored
 };
 static_assert(sizeof(SwapState) <= 1536, "lives in the tracker's mailboxes, which this layout leaves unused");
 
@@ -519,46 +523,40 @@ __device__ __forceinline__ int warp_best_bin(const unsigned *hist, int k1, int l
 }
 
 // Returns false when a wait ran out (the block then backs out like the other layouts).
-__device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st, uint32_t tmem_base, uint32_t tfull0,
-                                              uint32_t tempty0, volatile int *abort_flag, long long wait_limit,
-                                              int warp, int lane, int worker, int n_jobs, int n_workers) {
+// fail[2]: a wait ran out in a round of this parity.
+__device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st, volatile int *fail, uint32_t tmem_base,
+                                              uint32_t tfull0, uint32_t tempty0, volatile int *abort_flag,
+                                              long long wait_limit, int warp, int lane, int worker, int n_jobs,
+                                              int n_workers) {
     const int quarter = warp & 3;            // this warp's tensor-memory lanes: 32 * quarter ...
     const int tid128 = quarter * 32 + lane;
     const unsigned lt_mask = (1u << lane) - 1u;
+    const int n_pad = p.a_rows;              // accumulator columns per row group
+    const int n_chunks = n_pad / kSwapN;
     uint32_t acc = 0, acc_phase = 0;
     int round = 0;
     bool ok = true;
-    if (tid128 == 0) st->fail[0] = st->fail[1] = 0;
+    if (tid128 == 0) fail[0] = fail[1] = 0;
     for (int job = worker; job < n_jobs && ok; job += n_workers) {
         const int split = job % p.splits;    // one query tile: the job is the bank split
-        if (tid128 < kSwapN) {
+        if (tid128 < kSwapMax) {
             st->cnt[tid128] = 0;
             st->tau_bin[tid128] = 0;
             st->tau_sim[tid128] = -INFINITY;
-            st->floor_sim[tid128] = -INFINITY;
             st->tau_key[tid128] = 0;
             st->a_base[tid128] = -1;
-            st->mx[tid128] = 0;
         }
         epi_bar();
         int n_done = 0;
         for (int t = split; t < p.n_tiles; t += p.splits, ++n_done) {
-            if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) st->fail[round & 1] = 1;
+            if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, wait_limit)) fail[round & 1] = 1;
             epi_bar();
-            if (st->fail[round & 1]) { ok = false; break; }
+            if (fail[round & 1]) { ok = false; break; }
             ++round;
             tc_fence_after();
-            uint32_t v0[kSwapN], v1[kSwapN];   // this thread's row of group 0 and of group 1 against every query
+            // this thread's row of group 0 and of group 1 against sixteen queries at a time
+            uint32_t v0[kSwapN], v1[kSwapN];
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBlockN;
-            tmem_ld16_issue(t_addr, v0);
-            tmem_ld16_issue(t_addr + kSwapN, v1);
-            tmem_ld16_wait(v0);
-            tmem_ld16_wait(v1);
-            // the whole accumulator is in registers: hand it back
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             const int64_t row_a = (int64_t)t * kBlockN + tid128, row_b = row_a + kSubRows;
             const bool live_a = row_a < p.size && entry_live(p.live_bits, row_a);
             const bool live_b = row_b < p.size && entry_live(p.live_bits, row_b);
@@ -568,38 +566,52 @@ __device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st,
                 // The job's first 128 rows start the histogram off: their largest similarity anchors each
                 // query's window (whoever comes first), and those of them from window bin kBootBin up are
                 // counted before anything is filed (see the other layout's epilogue).
+#pragma unroll 1
+                for (int c = 0; c < n_chunks; ++c) {
+                    tmem_ld16_issue(t_addr + c * kSwapN, v0);
+                    tmem_ld16_wait(v0);
 #pragma unroll
-                for (int j = 0; j < kSwapN; ++j) {
-                    if (j < p.B) {
-                        const float x = __uint_as_float(v0[j]);
-                        const unsigned ob = (row_a < p.size && fabsf(x) <= 3.0e38f) ? ordered_bits(x + 0.0f) : 0u;
-                        const unsigned wm = __reduce_max_sync(0xffffffffu, ob);
-                        if (lane == 0 && wm) atomicMax(&st->mx[j], wm);
+                    for (int j = 0; j < kSwapN; ++j) {
+                        const int q = c * kSwapN + j;
+                        if (q < p.B) {
+                            const float x = __uint_as_float(v0[j]);
+                            const unsigned ob = (row_a < p.size && fabsf(x) <= 3.0e38f) ? ordered_bits(x + 0.0f) : 0u;
+                            const unsigned wm = __reduce_max_sync(0xffffffffu, ob);
+                            if (lane == 0 && wm) atomicMax(reinterpret_cast<unsigned *>(&st->cnt[q]), wm);
+                        }
                     }
                 }
                 epi_bar();
-                for (int j = quarter; j < p.B; j += 4) {
+                for (int q = quarter; q < p.B; q += 4) {
                     if (lane == 0) {
-                        int enc = __ldcg(p.anchor + j);
-                        if (enc == 0 && st->mx[j] != 0) {
-                            int prop = (int)(st->mx[j] >> kAbsShift) + kAbsHeadroom - (kHistBins - 1);
+                        const unsigned mx = (unsigned)st->cnt[q];
+                        int enc = __ldcg(p.anchor + q);
+                        if (enc == 0 && mx != 0) {
+                            int prop = (int)(mx >> kAbsShift) + kAbsHeadroom - (kHistBins - 1);
                             prop = prop < 0 ? 0 : (prop > kAbsBins - kHistBins ? kAbsBins - kHistBins : prop);
-                            const int got = atomicCAS(p.anchor + j, 0, prop + 1);
+                            const int got = atomicCAS(p.anchor + q, 0, prop + 1);
                             enc = got ? got : prop + 1;
                         }
-                        if (enc != 0) st->a_base[j] = enc - 1;
+                        if (enc != 0) st->a_base[q] = enc - 1;
                     }
                 }
                 epi_bar();
+                if (tid128 < kSwapMax) st->cnt[tid128] = 0;   // from here on: the lists' lengths
+#pragma unroll 1
+                for (int c = 0; c < n_chunks; ++c) {
+                    tmem_ld16_issue(t_addr + c * kSwapN, v0);
+                    tmem_ld16_wait(v0);
 #pragma unroll
-                for (int j = 0; j < kSwapN; ++j) {
-                    if (j < p.B) {
-                        const int ab = st->a_base[j];
-                        const float x = __uint_as_float(v0[j]);
-                        if (ab >= 0 && live_a && x >= from_ordered_bits((uint32_t)(ab + kBootBin) << kAbsShift)) {
-                            int bin = (int)(ordered_bits(x + 0.0f) >> kAbsShift) - ab;
-                            bin = bin > kHistBins - 1 ? kHistBins - 1 : bin;
-                            atomicAdd(p.hist + (size_t)j * kHistBins + bin, 1u);
+                    for (int j = 0; j < kSwapN; ++j) {
+                        const int q = c * kSwapN + j;
+                        if (q < p.B) {
+                            const int ab = st->a_base[q];
+                            const float x = __uint_as_float(v0[j]);
+                            if (ab >= 0 && live_a && x >= from_ordered_bits((uint32_t)(ab + kBootBin) << kAbsShift)) {
+                                int bin = (int)(ordered_bits(x + 0.0f) >> kAbsShift) - ab;
+                                bin = bin > kHistBins - 1 ? kHistBins - 1 : bin;
+                                atomicAdd(p.hist + (size_t)q * kHistBins + bin, 1u);
+                            }
                         }
                     }
                 }
@@ -609,66 +621,89 @@ __device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st,
             }
             // the thresholds: read before each of the first tiles, then before every kReadEvery-th
             if (n_done < kReadEvery || n_done % kReadEvery == 0) {
-                for (int j = quarter; j < p.B; j += 4) {
-                    const int ab = st->a_base[j];
+                for (int q = quarter; q < p.B; q += 4) {
+                    const int ab = st->a_base[q];
                     if (ab >= 0) {
-                        const int best = warp_best_bin(p.hist + (size_t)j * kHistBins, p.k1, lane);
-                        if (lane == 0 && best > st->tau_bin[j]) {
-                            st->tau_bin[j] = best;
-                            st->tau_sim[j] = fmaxf(st->floor_sim[j], from_ordered_bits((uint32_t)(ab + best) << kAbsShift));
+                        const int best = warp_best_bin(p.hist + (size_t)q * kHistBins, p.k1, lane);
+                        if (lane == 0 && best > st->tau_bin[q]) {
+                            st->tau_bin[q] = best;
+                            st->tau_sim[q] = fmaxf(key_sim(st->tau_key[q]), from_ordered_bits((uint32_t)(ab + best) << kAbsShift));
                         }
                     }
                 }
                 epi_bar();
             }
             // file what passes: one ballot per query and row group, the list's slots claimed per warp
-            auto file_one = [&](uint32_t bits, int64_t row, bool live, int j) {
+            auto file_one = [&](uint32_t bits, int64_t row, bool live, int q, float cheap) {
                 const float sv = __uint_as_float(bits);
-                bool pass = live && sv >= st->tau_sim[j];
+                bool pass = live && sv >= cheap;
+                // (nearly every ballot of the cheap test comes back empty)
+                if (!__any_sync(0xffffffffu, pass)) return;
                 uint64_t key = 0;
                 int bin = 0;
-                const int ab = st->a_base[j];
+                const int ab = st->a_base[q];
                 if (pass) {
                     key = make_key(sv, (int32_t)row);
                     if (ab >= 0) {
                         bin = (int)(ordered_bits(sv + 0.0f) >> kAbsShift) - ab;
                         bin = bin < 0 ? 0 : (bin > kHistBins - 1 ? kHistBins - 1 : bin);
                     }
-                    pass = key > st->tau_key[j] && bin >= st->tau_bin[j];
+                    pass = key > st->tau_key[q] && bin >= st->tau_bin[q];
                 }
                 const unsigned m = __ballot_sync(0xffffffffu, pass);
                 if (m) {
                     const int first = __ffs(m) - 1;
                     int base = 0;
-                    if (lane == first) base = atomicAdd(&st->cnt[j], __popc(m));
+                    if (lane == first) base = atomicAdd(&st->cnt[q], __popc(m));
                     base = __shfl_sync(0xffffffffu, base, first);
                     if (pass) {
-                        p.cand[((size_t)split * kBlockM + j) * kMmaCandCap + base + __popc(m & lt_mask)] = key;
+                        p.cand[((size_t)split * kBlockM + q) * kMmaCandCap + base + __popc(m & lt_mask)] = key;
                         // (entries of the counted first rows from kBootBin up are in the counters already)
                         if (ab >= 0 && (bin < skip_from || row >= counted_end))
-                            atomicAdd(p.hist + (size_t)j * kHistBins + bin, 1u);
+                            atomicAdd(p.hist + (size_t)q * kHistBins + bin, 1u);
                     }
                 }
             };
+#pragma unroll 1
+            for (int c = 0; c < n_chunks; ++c) {
+                tmem_ld16_issue(t_addr + c * kSwapN, v0);
+                tmem_ld16_issue(t_addr + n_pad + c * kSwapN, v1);
+                tmem_ld16_wait(v0);
+                tmem_ld16_wait(v1);
+                if (c == n_chunks - 1) {
+                    // the whole accumulator has been read: hand it back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                }
+                // the chunk's sixteen cheap thresholds in one trip to shared memory
+                float cheap[kSwapN];
 #pragma unroll
-            for (int j = 0; j < kSwapN; ++j) {
-                if (j < p.B) {
-                    file_one(v0[j], row_a, live_a, j);
-                    file_one(v1[j], row_b, live_b, j);
+                for (int j4 = 0; j4 < kSwapN / 4; ++j4) {
+                    const float4 f = *reinterpret_cast<const float4 *>(&st->tau_sim[c * kSwapN + 4 * j4]);
+                    cheap[4 * j4] = f.x; cheap[4 * j4 + 1] = f.y; cheap[4 * j4 + 2] = f.z; cheap[4 * j4 + 3] = f.w;
+                }
+#pragma unroll
+                for (int j = 0; j < kSwapN; ++j) {
+                    const int q = c * kSwapN + j;
+                    if (q < p.B) {
+                        file_one(v0[j], row_a, live_a, q, cheap[j]);
+                        file_one(v1[j], row_b, live_b, q, cheap[j]);
+                    }
                 }
             }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             // a list that the next tile could overflow (256 rows may all pass) is cut back to its best k1
             epi_bar();
-            for (int j = quarter; j < p.B; j += 4) {
-                const int n = st->cnt[j];
+            for (int q = quarter; q < p.B; q += 4) {
+                const int n = st->cnt[q];
                 if (n > kMmaCandCap - kBlockN) {
-                    const uint64_t kth = warp_select_topk(p.cand + ((size_t)split * kBlockM + j) * kMmaCandCap, n, p.k1);
+                    const uint64_t kth = warp_select_topk(p.cand + ((size_t)split * kBlockM + q) * kMmaCandCap, n, p.k1);
                     if (lane == 0) {
                         if (p.dev) atomicAdd(p.dev + kDevCutbacks, 1u);
-                        st->cnt[j] = p.k1;
-                        st->tau_key[j] = kth;
-                        st->floor_sim[j] = key_sim(kth);
-                        st->tau_sim[j] = fmaxf(st->tau_sim[j], st->floor_sim[j]);
+                        st->cnt[q] = p.k1;
+                        st->tau_key[q] = kth;
+                        st->tau_sim[q] = fmaxf(st->tau_sim[q], key_sim(kth));
                     }
                 }
             }
@@ -866,9 +901,9 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                     const uint64_t b_desc = smem_desc(s_addr + sl * (kSubRows * 128));
 #pragma unroll
                                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                                        if (kSwap)   // bank rows on the lanes, row group g in columns [16 g, 16 g + 16)
-                                            umma_bf16(d_tmem + g * kSwapN, b_desc + (uint64_t)(2 * k), a_desc + (uint64_t)(2 * k),
-                                                      (kc > 0 || k > 0) ? 1u : 0u, kInstrDescSwap);
+                                        if (kSwap)   // bank rows on the lanes, row group g in columns [N g, N g + N), N = a_rows
+                                            umma_bf16(d_tmem + g * p.a_rows, b_desc + (uint64_t)(2 * k), a_desc + (uint64_t)(2 * k),
+                                                      (kc > 0 || k > 0) ? 1u : 0u, instr_desc_swap(p.a_rows));
                                         else
                                             umma_bf16(d_tmem + g * kSubRows, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
                                                       (kc > 0 || k > 0) ? 1u : 0u, idesc);
@@ -910,7 +945,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         pdl_wait();
         if constexpr (kSwap) {
             SwapState *st = reinterpret_cast<SwapState *>(reinterpret_cast<unsigned char *>(bars) + 256);
-            swap_epilogue(p, st, tmem_base, tfull0, tempty0, abort_flag, wait_limit, warp, lane, worker, n_jobs, n_workers);
+            swap_epilogue(p, st, reinterpret_cast<volatile int *>(tmem_slot + 6), tmem_base, tfull0, tempty0, abort_flag,
+                          wait_limit, warp, lane, worker, n_jobs, n_workers);
             __syncwarp();
             if (lane == 0) atomicAdd(const_cast<int *>(epi_done), 1);
         } else {
@@ -1467,8 +1503,8 @@ struct SmemPlan {
 
 SmemPlan smem_plan(int B, int d) {
     SmemPlan sp;
-    // up to kSwapN queries of whole slices go to the swapped layout, whose query tile has kSwapN rows
-    const int rows = (B <= kSwapN && d % kBlockK == 0) ? kSwapN : (B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM);
+    // up to kSwapMax queries of whole slices go to the swapped layout, whose query tile is padded to 16 rows
+    const int rows = (B <= kSwapMax && d % kBlockK == 0) ? swap_n(B) : (B < kBlockM ? ((B + 7) / 8) * 8 : kBlockM);
     const size_t a_bytes = (size_t)rows * ((d + kBlockK - 1) / kBlockK * kBlockK) * 2;
     const size_t budget = kSmemMax - kSmemFixed;
     if (B <= kBlockM && a_bytes + 3 * (size_t)kBBytes <= budget) {
@@ -1729,7 +1765,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
         // attribute was seen, on B200 with driver 580, to run past its griddepcontrol.wait while its
         // predecessor was still running, so the paired scan is launched in plain stream order.)
         err = launch_kernel(map_q, map_bank, p, pl.grid, smem_bytes, p.abs_hist && !pl.pair && !ev_start,
-                            pl.pair != 0, stream, !pl.pair && p.b3d && B <= kSwapN);
+                            pl.pair != 0, stream, !pl.pair && p.b3d && B <= kSwapMax);
     if (err != cudaSuccess) return err;
     ++*launches;
     if (ev_stop) err = cudaEventRecord(ev_stop, stream);
