@@ -237,6 +237,10 @@ def _random_case(evk, n, d, b, k1, k2, w, seed, capacity=None, scoring=None):
     (300, 64, 130, 16, 4),       # two query tiles, the second nearly empty; bank just over one tile
     (66000, 128, 150, 512, 32),  # sampled thresholds, two query tiles, widest pool of the tensor path
     (40000, 128, 330, 96, 8),    # three query tiles: the second pair of blocks has one tile of queries only
+    (90000, 128, 16, 48, 6),     # the last batch size of one chunk of queries on the N side (bank rows on the lanes)
+    (90000, 192, 17, 48, 6),     # ... two chunks, the second with one query; three 64-column slices
+    (90000, 64, 32, 200, 9),     # ... the largest batch of that layout
+    (90000, 64, 33, 200, 9),     # the first batch with the queries back on the M side
 ])
 def test_edge_shapes(evk, n, d, b, k1, k2, scoring):
     _random_case(evk, n, d, b, k1, k2, 0.5, seed=n, scoring=scoring)
