@@ -31,6 +31,12 @@
 // With two or more query tiles, blocks run in clusters of two (cta_group::2): a pair shares
 // one 256-query x 256-row tile, each block loading its own queries and half of the bank slice.
 //
+// Up to 32 queries take the same pipeline with the operands' roles swapped (see kSwapN): the bank
+// rows sit on the accumulator's lanes (M = 128) and the queries on its columns, padded to 16 or 32
+// instead of to 64; a thread of the epilogue then owns a bank row, and what belongs to a query lives
+// in shared memory (swap_epilogue).  The scan is bound by HBM in either layout; the swapped one
+// spends a quarter to a half of the tensor work, which under the board's power cap is SM clock.
+//
 // A bank tile is 256 consecutive entries; the queries sit on the accumulator's
 // lanes so that the per-query threshold test costs one register compare and no
 // cross-thread traffic.  The work of a launch is a grid of jobs (query tile,
@@ -47,7 +53,8 @@
 // small histogram in global memory over the similarity range above its starting
 // threshold; every survivor is counted in it, and a threshold is raised to the highest bin
 // edge that was seen with k1 survivors at or above it.  With one query tile the scan runs
-// at HBM speed and each epilogue thread reads its query's counters before every tile; with
+// at HBM speed and each epilogue thread reads its query's counters before each of the first tiles and then
+// before every fourth; with
 // more, the tensor cores set the pace, the thread reads them itself only for the first
 // tiles of a job and the tracker warp takes over.  Counters only grow, so whatever mix of
 // old and new values a reader sees undercounts, and a threshold derived from it still has
