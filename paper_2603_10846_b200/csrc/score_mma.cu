@@ -510,10 +510,9 @@ static_assert(sizeof(SwapState) <= 1536, "lives in the tracker's mailboxes, whic
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Highest bin of the histogram with k1 counted entries at or above it (0: none yet); the whole warp
-// reads the 64 counters, two per lane.
-__device__ __forceinline__ int warp_best_bin(const unsigned *hist, int k1, int lane) {
-    const uint2 c = __ldcg(reinterpret_cast<const uint2 *>(hist) + lane);
+// Highest bin of a histogram with k1 counted entries at or above it (0: none yet), from the 64 counters
+// held two per lane.
+__device__ __forceinline__ int warp_best_bin(uint2 c, int k1, int lane) {
     int own = (int)(c.x + c.y), incl = own;   // incl: this lane's counters and all higher ones
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -589,8 +588,10 @@ __device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st,
                     }
                 }
                 epi_bar();
-                for (int q = quarter; q < p.B; q += 4) {
-                    if (lane == 0) {
+                {
+                    // one lane per query of this warp's share (quarter, quarter + 4, ...)
+                    const int q = quarter + 4 * lane;
+                    if (q < p.B) {
                         const unsigned mx = (unsigned)st->cnt[q];
                         int enc = __ldcg(p.anchor + q);
                         if (enc == 0 && mx != 0) {
@@ -628,13 +629,26 @@ __device__ __forceinline__ bool swap_epilogue(const MmaParams &p, SwapState *st,
             }
             // the thresholds: read before each of the first tiles, then before every kReadEvery-th
             if (n_done < kReadEvery || n_done % kReadEvery == 0) {
-                for (int q = quarter; q < p.B; q += 4) {
-                    const int ab = st->a_base[q];
-                    if (ab >= 0) {
-                        const int best = warp_best_bin(p.hist + (size_t)q * kHistBins, p.k1, lane);
-                        if (lane == 0 && best > st->tau_bin[q]) {
-                            st->tau_bin[q] = best;
-                            st->tau_sim[q] = fmaxf(key_sim(st->tau_key[q]), from_ordered_bits((uint32_t)(ab + best) << kAbsShift));
+                // this warp's queries (quarter, quarter + 4, ...): all their counters are asked for before the
+                // first answer is looked at, one trip to L2 instead of one per query
+                uint2 ctr[kSwapMax / 4];
+#pragma unroll
+                for (int i = 0; i < kSwapMax / 4; ++i) {
+                    const int q = quarter + 4 * i;
+                    ctr[i] = (q < p.B) ? __ldcg(reinterpret_cast<const uint2 *>(p.hist + (size_t)q * kHistBins) + lane)
+                                       : make_uint2(0u, 0u);
+                }
+#pragma unroll
+                for (int i = 0; i < kSwapMax / 4; ++i) {
+                    const int q = quarter + 4 * i;
+                    if (q < p.B) {
+                        const int ab = st->a_base[q];
+                        if (ab >= 0) {
+                            const int best = warp_best_bin(ctr[i], p.k1, lane);
+                            if (lane == 0 && best > st->tau_bin[q]) {
+                                st->tau_bin[q] = best;
+                                st->tau_sim[q] = fmaxf(key_sim(st->tau_key[q]), from_ordered_bits((uint32_t)(ab + best) << kAbsShift));
+                            }
                         }
                     }
                 }
