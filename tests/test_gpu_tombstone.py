@@ -43,7 +43,9 @@ def _retrieve(evk, mem, queries, stage, k1, k2, w):
 
 
 @pytest.mark.parametrize("n,d,b,k1,k2", [
-    (30000, 256, 7, 64, 8),        # one query tile, thresholds started off by the scan itself
+    (30000, 256, 7, 64, 8),        # one query tile, thresholds started off by the scan itself (bank rows on the lanes)
+    (30000, 256, 50, 64, 8),       # ... queries on the lanes, resident in shared memory
+    (30000, 1024, 100, 64, 8),     # ... queries on the lanes, streamed through the ring
     (70000, 128, 200, 96, 8),      # a pair of query tiles: sampled thresholds, some sampled rows dropped
     (900, 64, 3, 40, 5),           # a small bank
 ])
