@@ -608,10 +608,12 @@ def test_tensor_path_candidate_lists_overflow_and_are_cut_back(evk):
     parity.check_retrieve(host_bits(bank2), host_bits(queries), q_tab[0], k1, 10, 0.5, out2, sample=[0, 1, 1999])
 
 
-def test_few_queries_lists_overflow_and_are_cut_back(evk):
-    # up to 16 queries take the layout with the bank rows on the accumulator lanes; a bank sorted against
-    # the scan for query 0 makes every row of every tile pass, so that its lists fill and are cut back
-    n, d, b, k1 = 250000, 64, 3, 100
+@pytest.mark.parametrize("b", [3, 40])
+def test_one_query_tile_lists_overflow_and_are_cut_back(evk, b):
+    # a bank sorted against the scan for query 0 makes every row of every tile pass, so that its lists fill
+    # and are cut back: 3 queries in the layout with the bank rows on the accumulator lanes, 40 in the one
+    # with the queries there
+    n, d, k1 = 250000, 64, 100
     bank = synth.gaussian_unit(n, d, 97, DEV)
     queries = synth.gaussian_unit(b, d, 98, DEV)
     order = torch.argsort((bank.float() @ queries[:1].float().T).squeeze(1))
@@ -621,7 +623,8 @@ def test_few_queries_lists_overflow_and_are_cut_back(evk):
     before = evk.evk_mem_stats(mem)["list_cutbacks"]
     out = run_retrieve(evk, mem, queries, 0, k1, 10, 0.5)
     assert evk.evk_mem_stats(mem)["list_cutbacks"] > before
-    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, 10, 0.5, out)
+    ep, ef = parity.check_retrieve(host_bits(bank), host_bits(queries), q_tab[0], k1, 10, 0.5, out,
+                                   sample=[0, 1, b - 1] + sample_of(b, 5, seed=4))
     assert ep == 1.0 and ef == 1.0
 
 
