@@ -1357,11 +1357,14 @@ constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = kMmaSample / kSelThreads;
 constexpr int kSelBins = 1024;
 
-__global__ void __launch_bounds__(kSelThreads)
+// (The samples are kept in shared memory, not in registers: at 64 registers a thread only four blocks fit
+// an SM and 1,024 queries took two waves.)
+__global__ void __launch_bounds__(kSelThreads, 8)
 sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, int k1, float *__restrict__ tau0,
                         float2 *__restrict__ range, unsigned *__restrict__ hist_out,
                         const uint32_t *__restrict__ live_bits, int64_t sample_stride) {
     __shared__ int bins[kSelBins];
+    __shared__ float sv[kMmaSample];
     __shared__ float red_lo[kSelThreads / 32], red_hi[kSelThreads / 32];
     __shared__ int red_cnt[kSelThreads / 32];
     __shared__ int chosen;
@@ -1372,7 +1375,6 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
     for (int i = tid; i < kSelBins; i += kSelThreads) bins[i] = 0;
     if (tid == 0) chosen = 0;
     // this thread's samples; a non-finite similarity counts as the lowest value
-    float v[kSelPerThread];
     float lo = INFINITY, hi = -INFINITY;
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j) {
@@ -1381,7 +1383,7 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
         // a non-finite similarity, or a sampled entry that has been dropped from the memory, counts as
         // the lowest value: it cannot vouch for a threshold
         if (i < n_sample && (!(fabsf(x) <= 3.0e38f) || !entry_live(live_bits, (int64_t)i * sample_stride))) x = -3.0e38f;
-        v[j] = x;
+        sv[tid + j * kSelThreads] = x;   // read back by this thread alone
         if (i < n_sample) {
             lo = fminf(lo, x);
             hi = fmaxf(hi, x);
@@ -1404,14 +1406,13 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
     }
     float scale = (float)kSelBins / (hi - lo);
     if (!(scale > 0.0f) || !(scale < 3.0e38f)) scale = 0.0f;   // no spread: everything in bin 0
-    int my_bin[kSelPerThread];
-#pragma unroll
-    for (int j = 0; j < kSelPerThread; ++j) {
-        int b = (int)((v[j] - lo) * scale);
-        b = b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
-        my_bin[j] = b;
-        if (tid + j * kSelThreads < n_sample) atomicAdd(&bins[b], 1);
-    }
+    auto bin_of = [&](float x) {
+        const int b = (int)((x - lo) * scale);
+        return b < 0 ? 0 : (b > kSelBins - 1 ? kSelBins - 1 : b);
+    };
+#pragma unroll 4
+    for (int j = 0; j < kSelPerThread; ++j)
+        if (tid + j * kSelThreads < n_sample) atomicAdd(&bins[bin_of(sv[tid + j * kSelThreads])], 1);
     __syncthreads();
     // thread t owns bins [4t, 4t+4); count of samples in its bins and in all higher ones
     int mine[4], sum = 0;
@@ -1445,9 +1446,11 @@ sample_threshold_kernel(const float *__restrict__ dense, int ld, int n_sample, i
     __syncthreads();
     const int b_min = chosen;
     float t = INFINITY;
-#pragma unroll
-    for (int j = 0; j < kSelPerThread; ++j)
-        if (tid + j * kSelThreads < n_sample && my_bin[j] >= b_min) t = fminf(t, v[j]);
+#pragma unroll 4
+    for (int j = 0; j < kSelPerThread; ++j) {
+        const float x = sv[tid + j * kSelThreads];
+        if (tid + j * kSelThreads < n_sample && bin_of(x) >= b_min) t = fminf(t, x);
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) t = fminf(t, __shfl_xor_sync(0xffffffffu, t, off));
     if (lane == 0) red_lo[warp] = t;   // last read of red_lo was before two barriers
