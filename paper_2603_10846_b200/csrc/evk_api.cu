@@ -326,6 +326,7 @@ int evk_retrieve(evk_mem *mem, const void *queries, int q_dtype, int32_t B, int 
             mem->stall_next = 0;
             plan.live_bits = mem->any_dropped ? mem->live_bits : nullptr;
             plan.dev = mem->dev;
+            plan.wait_queries = q_dtype == EVK_DTYPE_F32 ? 1 : 0;
             uint64_t *cand = nullptr;
             int *cand_cnt = nullptr;
             err = launch_score_mma(mem->bank, mem->size, mem->cfg.capacity, mem->cfg.d, q_bf16, B, k1, plan,

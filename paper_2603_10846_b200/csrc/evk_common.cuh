@@ -45,7 +45,10 @@ __device__ __forceinline__ bool entry_live(const uint32_t *live_bits, int64_t id
 
 // Per-bank words in device memory (the 256-byte block at the end of the arena).
 enum DevWord { kDevStatus = 0, kDevLive = 1, kDevFiledLo = 2, kDevFiledHi = 3, kDevCutbacks = 4, kDevLongestRun = 5,
-               kDevFlag = 6, kDevDropped = 7 };
+               kDevFlag = 6, kDevDropped = 7,
+               // rows [0, kDevRowsReady) of the bank are in memory: published by every insert once all its
+               // blocks have written theirs (kDevInsTicket counts them), read by the scan before it loads a tile
+               kDevRowsReady = 8, kDevInsTicket = 9 };
 
 // Claims one slot of a shared counter for every lane whose `want` is set, with a single atomic
 // per warp.  Every lane of the warp must call it; returns the lane's slot (undefined if !want).

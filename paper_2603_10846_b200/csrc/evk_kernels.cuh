@@ -52,6 +52,8 @@ struct MmaPlan {
     int stall;              // test aid, see evk_mem_inject_stall
     const uint32_t *live_bits;   // entries dropped from the memory are skipped (null: none ever was)
     uint32_t *dev;               // the bank's device words (counters), or null
+    int wait_queries;            // the query matrix comes out of the library's own conversion kernel, which may
+                                 // still be running when the scan starts (mma_plan sets 1, the cautious value)
 };
 bool mma_supported(int d, int k1);
 MmaPlan mma_plan(int64_t size, int B, int k1);

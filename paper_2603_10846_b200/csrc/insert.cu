@@ -72,6 +72,17 @@ insert_kernel(__nv_bfloat16 *__restrict__ dst, const void *__restrict__ src, int
         if (ids_out) ids_out[i] = (int32_t)(first + i);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(dev + kDevLive, (uint32_t)n);
+    // The last block to get here tells the scans that the rows are there.  (Inserts never overlap one
+    // another: each waits for the kernel before it, so the ticket counter is back at 0 for the next.)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(dev + kDevInsTicket, 1u) == gridDim.x - 1) {
+            dev[kDevInsTicket] = 0;
+            __threadfence();
+            atomicMax(dev + kDevRowsReady, (uint32_t)(first + n));
+        }
+    }
 }
 
 // ---- entries dropped from a live bank ------------------------------------------------------------

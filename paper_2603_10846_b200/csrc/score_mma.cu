@@ -134,6 +134,7 @@ struct MmaParams {
     int *anchor;        // [B] abs_hist: lowest bin of each query's histogram window + 1, 0 until the first block sets it
     const uint32_t *live_bits;   // entries dropped from the memory are skipped (null: none ever was)
     uint32_t *dev;      // the bank's device words: candidates filed and list cut-backs are counted there (or null)
+    int wait_queries;   // the queries come out of the library's conversion kernel: wait for it before loading them
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -159,6 +160,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait; false means the block is aborting.
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -847,6 +854,17 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // would let it go in between (4,096 queries over 6 GiB: 22.7 against 19.5 ms).
             const bool stream_once = kMode == 0 && (kPair ? p.n_qt <= 2 : p.n_qt == 1);
             const uint64_t bank_policy = l2_evict_first_policy();
+            // This kernel may have been started while the kernels before it still run: their blocks have said
+            // that dependents may be scheduled, not that they are done, and the same holds for the kernels
+            // before those.  Rows appended by an insert - even two calls ago - may not be in memory yet (seen on
+            // a bank of one tile: a third of 400 rounds of insert -> retrieve returned stale rows).  So a tile is
+            // loaded only once the bank's rows-ready word, which every insert publishes behind its last row,
+            // covers it: nearly all tiles at once (the scan streams while the merge, the update and the insert
+            // before it finish), the last one when that insert is done.  Without the word, and for queries that
+            // the library's own conversion kernel writes, no load is issued before griddepcontrol.wait.
+            if (p.wait_queries || !p.dev) pdl_wait();
+            int64_t rows_ready = p.dev ? (int64_t)ld_acquire_u32(p.dev + kDevRowsReady) : p.size;
+            if (kMode == 1) rows_ready = INT64_MAX;   // the sample pass is launched in plain stream order
             if (ok && p.a_resident && worker < n_jobs) {
                 a_armed = true;
                 mbar_arrive_expect_tx(afull, a_region);
@@ -856,6 +874,22 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int qt = kPair ? (job / p.splits) * 2 + (int)rank : job / p.splits;
                 const int split = job % p.splits;
                 for (int t = split; t < p.n_tiles && ok; t += p.splits) {
+                    {
+                        const int64_t tile_end = (int64_t)(t + 1) * kBlockN;
+                        const int64_t need = tile_end < p.size ? tile_end : p.size;
+                        if (rows_ready < need) {
+                            const long long t0 = clock64();
+                            while ((rows_ready = (int64_t)ld_acquire_u32(p.dev + kDevRowsReady)) < need) {
+                                if (*abort_flag || clock64() - t0 > wait_limit) {
+                                    *abort_flag = 1;
+                                    ok = false;
+                                    break;
+                                }
+                                __nanosleep(200);
+                            }
+                            if (!ok) break;
+                        }
+                    }
                     for (int u = 0; u < n_sub; ++u) {
                         if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                         const uint32_t s_dst = ring + stage * stage_bytes;
@@ -961,8 +995,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else if (warp < 6) {
         // ===== epilogue: thread = one query of the tile = one TMEM lane =====
-        // The thresholds, the histogram and the candidate lists belong to the kernels before this
-        // one; loads and MMAs of the first tiles run ahead while the epilogue waits for them.
+        // The thresholds, the histogram and the candidate lists belong to the kernels before this one.
         pdl_wait();
         if constexpr (kSwap) {
             SwapState *st = reinterpret_cast<SwapState *>(reinterpret_cast<unsigned char *>(bars) + 256);
@@ -1662,6 +1695,7 @@ MmaPlan mma_plan(int64_t size, int B, int k1) {
     pl.stall = 0;
     pl.live_bits = nullptr;
     pl.dev = nullptr;
+    pl.wait_queries = 1;
     return pl;
 }
 
@@ -1702,6 +1736,7 @@ cudaError_t launch_score_mma(const __nv_bfloat16 *bank, int64_t size, int64_t ca
     p.hist = hist;
     p.live_bits = pl.live_bits;
     p.dev = pl.dev;
+    p.wait_queries = pl.wait_queries;
     p.abs_hist = pl.pair ? 0 : 1;
     p.anchor = reinterpret_cast<int *>(tau0);   // the sampled thresholds' array, unused by such a scan
     // One query tile: the scan runs at HBM speed, a bank tile arrives every ~11 us and the epilogue

@@ -520,6 +520,35 @@ def test_kernels_of_one_stream_wait_for_one_another(evk, b, k2):
     assert np.array_equal(evk.evk_q_read(mem, 1).cpu().numpy().view(np.uint32), q_orc.view(np.uint32))
 
 
+@pytest.mark.parametrize("d,dtype", [(1024, torch.bfloat16), (64, torch.bfloat16), (2048, torch.float32)])
+def test_a_retrieval_sees_the_rows_appended_just_before_it(evk, d, dtype):
+    """The scan is launched so that it may start while the kernels before it still run (and those before
+    them: every kernel of the library lets its successor be scheduled at once).  Rows appended by the
+    insert just before it, or two calls ago, and fp32 queries, which the library converts in a kernel of its
+    own, must be loaded only once those kernels are done: on a bank of one or two tiles the first loads would
+    otherwise meet rows that are still being written (seen: a third of 400 rounds returned a stale
+    neighbour).  400 rounds of insert 16 rows -> retrieve them, nothing synchronises; the three cases run
+    in one process on purpose (recycled memory holds garbage where a row is not yet written)."""
+    n0, rounds, n_new = 40, 400, 16
+    mem = evk.evk_mem_create(d, n0 + rounds * n_new + 64)
+    evk.evk_mem_insert(mem, synth.gaussian_unit(n0, d, 1, DEV))
+    rows = synth.gaussian_unit(rounds * n_new, d, 2, DEV)
+    queries = rows.to(dtype)
+    outs = torch.empty((rounds, n_new), dtype=torch.int32, device=DEV)
+    sc = torch.empty((n_new, 1), dtype=torch.float32, device=DEV)
+    busy = torch.empty(1 << 28, dtype=torch.uint8, device=DEV)
+    torch.cuda.synchronize()
+    for _ in range(4):
+        busy.zero_()          # the launches below queue up behind this and then run back to back
+    for r in range(rounds):
+        evk.evk_mem_insert(mem, rows[r * n_new:(r + 1) * n_new])
+        evk.evk_retrieve(mem, queries[r * n_new:(r + 1) * n_new], 0, 8, 1, 0.0, out=(outs[r].view(n_new, 1), sc))
+    torch.cuda.synchronize()
+    assert evk.evk_last_status(mem) == 0
+    want = (torch.arange(rounds * n_new, device=DEV, dtype=torch.int32) + n0).view(rounds, n_new)
+    assert torch.equal(outs, want)
+
+
 def test_host_buffer_calls_check_arguments_before_copying(evk):
     # a refused call enqueues nothing: no kernel is launched, the outputs keep their contents
     n, d, b, k1, k2 = 5000, 128, 4, 32, 4
