@@ -864,6 +864,8 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // the library's own conversion kernel writes, no load is issued before griddepcontrol.wait.
             if (p.wait_queries || !p.dev) pdl_wait();
             int64_t rows_ready = p.dev ? (int64_t)ld_acquire_u32(p.dev + kDevRowsReady) : p.size;
+            // (the rows were written with ordinary stores and are read by bulk tensor copies: order the two proxies)
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             if (kMode == 1) rows_ready = INT64_MAX;   // the sample pass is launched in plain stream order
             if (ok && p.a_resident && worker < n_jobs) {
                 a_armed = true;
@@ -888,6 +890,7 @@ score_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 __nanosleep(200);
                             }
                             if (!ok) break;
+                            asm volatile("fence.proxy.async.global;" ::: "memory");
                         }
                     }
                     for (int u = 0; u < n_sub; ++u) {
