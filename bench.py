@@ -38,9 +38,9 @@ UNIT = "queries/s"
 NOMINAL_HBM_GBS = 8000.0          # the HBM3e figure the bandwidth target is quoted against
 # DRAM bytes (read + written) per scanned bank entry of width 1024, from one ncu capture of the
 # scan kernel; see TRAFFIC_SOURCE.  The bank is read once per launch, so traffic grows with the rows.
-SCAN_DRAM_BYTES_PER_ENTRY = 541.51e6 / 262147
+SCAN_DRAM_BYTES_PER_ENTRY = 541.86e6 / 262147
 TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one score_mma_kernel launch, "
-                  "262,147 rows x 1024 bf16 (512 MiB), 64 queries, k1=128: 537.81 + 3.70 MB = 2,065.7 B per entry "
+                  "262,147 rows x 1024 bf16 (512 MiB), 64 queries, k1=128: 537.81 + 4.04 MB = 2,067.0 B per entry "
                   "against 2,048 B algorithmic; scaled by the rows one launch scans")
 
 
